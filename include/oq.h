@@ -1,0 +1,142 @@
+/*
+ * liboq -- B200 (sm_100a) runtime hot path of an OrbitQuant quantized linear layer.
+ *
+ * One quantized linear layer y = W x (paper Eq. 1) is computed as
+ *
+ *     offline   Pi_d  <- RPBH(d)                       oq_make_rpbh        (Eq. 9, Algorithm 1 "Offline")
+ *               C^(d,b) <- LloydMax(d, b)              oq_build_codebook   (Eq. 2-3, Sec. 4.5)
+ *               W^' <- diag(r') Q_bw(rows of W Pi^T)   oq_quantize_weights (Eq. 4-6)
+ *     online    x^' <- s Q_ba(Pi x / (s + eps))        oq_rotate_quantize_act (Eq. 7-8, Algorithm 1 "Online")
+ *               y   <- W^' x^'                         oq_qlinear          (Sec. 4.3: the rotation cancels)
+ *
+ * Conventions
+ *   - Plain C ABI.  Every call returns an OQ_* status; oq_last_error() gives a message for the last
+ *     failure on the calling thread.  Nothing throws across the boundary.
+ *   - "dev" pointers are CUDA device pointers on the current device, owned by the caller (for example a
+ *     PyTorch tensor's data_ptr()).  "host" pointers are ordinary host memory.  The library allocates
+ *     only the small tables that belong to an oq_rpbh handle (permutation and signs, < 128 KB, uploaded on
+ *     first use on the device that is current at that moment and freed by oq_rpbh_destroy).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Kernel launches are
+ *     asynchronous on that stream; argument validation happens on the host before any launch.
+ *   - Matrices are row-major.  X is [n_tokens][ldx] bf16, W is [m][ldw] bf16 (the layout of a linear
+ *     layer's weight, W in R^{m x d}); ld* are in elements.
+ *   - Quantized operands are PACKED: `bits` bits per coordinate on the wire, in a layout private to the
+ *     library (oq_packed_bytes gives the sizes; oq_unpack_indices recovers the logical level indices,
+ *     numbered 0 .. 2^bits-1 in ascending order of the level, in rotated-coordinate order).
+ *   - There is no CPU fallback: a call that needs the GPU fails with OQ_ERR_CUDA if no device is usable.
+ */
+#ifndef OQ_H_
+#define OQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  OQ_OK = 0,
+  OQ_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, mismatching handles */
+  OQ_ERR_UNSUPPORTED = 2,    /* dim / block / bits outside what the kernels implement */
+  OQ_ERR_ALIGNMENT = 3,      /* pointer not 16-byte aligned or leading dimension not a multiple of 8 */
+  OQ_ERR_CUDA = 4,           /* a CUDA runtime call failed (message holds the CUDA error string) */
+  OQ_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait gave up (see oq_device_status) */
+  OQ_ERR_NOMEM = 6           /* workspace too small / allocation failed */
+};
+
+enum { OQ_BF16 = 0, OQ_F32 = 1 }; /* output element type of oq_qlinear */
+
+typedef struct oq_codebook oq_codebook; /* Lloyd-Max codebook C^(d,b): host tables only */
+typedef struct oq_rpbh oq_rpbh;         /* RPBH rotation Pi_d: permutation + signs (host, and device on first use) */
+
+/* ---- offline constructors (host arithmetic in fp64; usable without a GPU) ------------------------- */
+
+/* Lloyd-Max codebook of 2^bits levels for the coordinate marginal f_dim of a random unit vector
+ * (Eq. 2: f_d(t) ~ (1 - t^2)^((d-3)/2) on [-1,1]; Eq. 3: nearest-level map).  The exact f_dim is used,
+ * not its Gaussian approximation.  dim >= 16, bits in 1..4.  *out is owned by the caller
+ * (oq_codebook_destroy).  Errors: OQ_ERR_INVALID_ARG, OQ_ERR_UNSUPPORTED. */
+int oq_build_codebook(int dim, int bits, oq_codebook** out);
+
+/* Copies the tables out (any pointer may be NULL): centroids[2^bits] ascending (fp64),
+ * boundaries[2^bits-1] = midpoints of adjacent levels (fp64), boundaries_f32 = those rounded once to
+ * fp32, centroids_bf16 = levels rounded fp64 -> fp32 -> bf16 (the values the GEMM decodes to). */
+int oq_codebook_get(const oq_codebook* cb, double* centroids, double* boundaries,
+                    float* boundaries_f32, uint16_t* centroids_bf16);
+int oq_codebook_dim(const oq_codebook* cb);
+int oq_codebook_bits(const oq_codebook* cb);
+void oq_codebook_destroy(oq_codebook* cb);
+
+/* Randomized permuted block-Hadamard rotation Pi_d = blkdiag(H_h D_1, ..., H_h D_{d/h}) P_pi (Eq. 9):
+ * uniform permutation pi (applied first, as a gather: (P x)_k = x[pi(k)]), Rademacher signs indexed by
+ * the position after the permutation, Sylvester-ordered Walsh-Hadamard blocks scaled by 1/sqrt(h).
+ * The draw is deterministic in (dim, block, seed): SplitMix64 with initial state
+ * seed ^ (dim << 32) ^ block, Fisher-Yates from the top with rejection sampling, then one 64-bit word
+ * per 64 signs (bit set = -1).  block: power of two, divides dim; dim < 65536. */
+int oq_make_rpbh(int dim, int block, uint64_t seed, oq_rpbh** out);
+/* perm[dim] (int32) and signs[dim] (int8, +1 / -1); either may be NULL. */
+int oq_rpbh_get(const oq_rpbh* r, int32_t* perm, int8_t* signs);
+int oq_rpbh_dim(const oq_rpbh* r);
+int oq_rpbh_block(const oq_rpbh* r);
+void oq_rpbh_destroy(oq_rpbh* r);
+
+/* ---- sizes -------------------------------------------------------------------------------------------- */
+
+/* Bytes of the packed index matrix of `rows` rows of `dim` coordinates at `bits` bits each, and the
+ * pitch of one row (a multiple of 16 bytes).  dim must be a multiple of 128; bits in {2,3,4}. */
+int oq_packed_bytes(int rows, int dim, int bits, size_t* idx_bytes, size_t* row_pitch_bytes);
+
+/* ---- GPU entry points ---------------------------------------------------------------------------------- */
+
+/* Online activation quantization, one fused pass per token (Eq. 7-8, Algorithm 1 lines "Online"):
+ * x' = Pi x, s = ||x'||_2, idx_k = level of C^(d,b_a) nearest to x'_k / (s + 1e-10).
+ *   X_bf16     dev  [n_tokens][ldx] bf16, read only
+ *   Xq_idx     dev  packed indices, oq_packed_bytes(n_tokens, dim, bits) bytes, written
+ *   Xq_norm    dev  [n_tokens] fp32, s per token, written
+ *   dbg_rotated dev [n_tokens][dim] fp32 or NULL; when given, receives x' (test hook; slows the kernel)
+ * s is the norm of the raw row (equal to ||Pi x|| because Pi is orthogonal), accumulated in fp32.
+ * A zero token gives s = 0 and the lower middle level everywhere.  n_tokens may be 0 (no launch).
+ * Requires dim == rpbh dim == codebook dim, dim % 128 == 0, ldx >= dim, ldx % 8 == 0, 16-byte aligned
+ * pointers.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA. */
+int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                           const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated,
+                           void* stream);
+
+/* Offline weight quantization, run on the GPU (Eq. 4-6): the same pass applied to the m rows of W
+ * (row i of W Pi^T is Pi w_i); the row norm r'_i is stored in bf16 (Sec. 4.2).
+ *   W_bf16 dev [m][ldw] bf16; Wq_idx dev packed (oq_packed_bytes(m, dim, bits)); Wq_norm_bf16 dev [m] bf16.
+ * The GEMM tiles weights in groups of 128 rows; rows beyond m need not exist (they are never read). */
+int oq_quantize_weights(const void* W_bf16, int m, int dim, int ldw, const oq_rpbh* rot,
+                        const oq_codebook* cb_w, void* Wq_idx, void* Wq_norm_bf16, void* dbg_rotated,
+                        void* stream);
+
+/* Quantized linear layer on packed operands (the product W^' x^' of Sec. 4.3 with Eq. 6 and Eq. 8):
+ *   Y[n][i] = s_n * r'_i * sum_k C_a[idxA[n][k]] * C_w[idxW[i][k]]
+ * Levels are decoded to bf16 in shared memory, contracted on the tensor cores with fp32 accumulation,
+ * and both norms are applied in the epilogue (acc * s_n * r'_i, two fp32 multiplies in that order, then
+ * one rounding when Y is bf16).
+ *   Xq_idx, Xq_norm  dev  as written by oq_rotate_quantize_act with cb_a
+ *   Wq_idx, Wq_norm_bf16 dev as written by oq_quantize_weights with cb_w
+ *   Y dev [n_tokens][ldy] of y_dtype (OQ_BF16 or OQ_F32), written; ldy >= m, ldy % 8 == 0
+ * Requires the two codebooks to have the same dim (= dim), dim % 128 == 0, m % 8 == 0.
+ * n_tokens == 0 or m == 0 launches nothing.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA. */
+int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
+               const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim,
+               void* Y, int ldy, int y_dtype, void* stream);
+
+/* Test helper: expand packed indices to one byte per coordinate, out dev [rows][dim] uint8, logical level
+ * numbers in rotated-coordinate order. */
+int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream);
+
+/* Synchronises the device and reports (then clears) the device-side status word: 0 when every bounded
+ * wait inside the kernels completed, otherwise a code saying which wait gave up.  Returns OQ_OK or
+ * OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
+int oq_device_status(int* status);
+
+const char* oq_last_error(void);
+const char* oq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OQ_H_ */

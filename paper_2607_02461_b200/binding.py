@@ -1,0 +1,184 @@
+"""Thin ctypes binding of liboq.so: same names as the C entry points, argument marshalling only.
+
+Device buffers are torch CUDA tensors (torch owns memory and streams); every step of the path runs in
+the library's kernels.  There is no fallback: if liboq.so is missing or a call fails, OqError is raised.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liboq.so")
+_lib = None
+
+OQ_BF16, OQ_F32 = 0, 1
+STATUS_NAMES = {0: "OQ_OK", 1: "OQ_ERR_INVALID_ARG", 2: "OQ_ERR_UNSUPPORTED", 3: "OQ_ERR_ALIGNMENT",
+                4: "OQ_ERR_CUDA", 5: "OQ_ERR_DEVICE_TIMEOUT", 6: "OQ_ERR_NOMEM"}
+
+
+class OqError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+def lib():
+    """Loads liboq.so (built in-tree by paper_2607_02461_b200.build); fails loudly when absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise OqError(4, f"{_LIB_PATH} not found: run `python -m paper_2607_02461_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        vp, i, u64, sz = C.c_void_p, C.c_int, C.c_uint64, C.c_size_t
+        pp = C.POINTER(C.c_void_p)
+        sig = {
+            "oq_build_codebook": (i, [i, i, pp]),
+            "oq_codebook_get": (i, [vp, vp, vp, vp, vp]),
+            "oq_codebook_dim": (i, [vp]), "oq_codebook_bits": (i, [vp]), "oq_codebook_destroy": (None, [vp]),
+            "oq_make_rpbh": (i, [i, i, u64, pp]),
+            "oq_rpbh_get": (i, [vp, vp, vp]),
+            "oq_rpbh_dim": (i, [vp]), "oq_rpbh_block": (i, [vp]), "oq_rpbh_destroy": (None, [vp]),
+            "oq_packed_bytes": (i, [i, i, i, C.POINTER(sz), C.POINTER(sz)]),
+            "oq_rotate_quantize_act": (i, [vp, i, i, i, vp, vp, vp, vp, vp, vp]),
+            "oq_quantize_weights": (i, [vp, i, i, i, vp, vp, vp, vp, vp, vp]),
+            "oq_qlinear": (i, [vp, vp, i, vp, vp, vp, i, vp, i, vp, i, i, vp]),
+            "oq_unpack_indices": (i, [vp, i, i, i, vp, vp]),
+            "oq_device_status": (i, [C.POINTER(i)]),
+            "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
+        }
+        for name, (res, args) in sig.items():
+            if hasattr(L, name):
+                f = getattr(L, name)
+                f.restype, f.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(code):
+    if code != 0:
+        raise OqError(code, lib().oq_last_error().decode())
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Codebook:
+    """Owns an oq_codebook handle."""
+
+    def __init__(self, dim, bits):
+        h = C.c_void_p()
+        _check(lib().oq_build_codebook(dim, bits, C.byref(h)))
+        self.handle, self.dim, self.bits = h, dim, bits
+        L = 1 << bits
+        self.centroids = np.zeros(L, np.float64)
+        self.boundaries = np.zeros(L - 1, np.float64)
+        self.boundaries_f32 = np.zeros(L - 1, np.float32)
+        self.centroids_bf16_bits = np.zeros(L, np.uint16)
+        _check(lib().oq_codebook_get(h, self.centroids.ctypes.data, self.boundaries.ctypes.data,
+                                     self.boundaries_f32.ctypes.data, self.centroids_bf16_bits.ctypes.data))
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.oq_codebook_destroy(self.handle)
+            self.handle = None
+
+
+class Rpbh:
+    """Owns an oq_rpbh handle."""
+
+    def __init__(self, dim, block, seed):
+        h = C.c_void_p()
+        _check(lib().oq_make_rpbh(dim, block, seed, C.byref(h)))
+        self.handle, self.dim, self.block, self.seed = h, dim, block, seed
+        self.perm = np.zeros(dim, np.int32)
+        self.signs = np.zeros(dim, np.int8)
+        _check(lib().oq_rpbh_get(h, self.perm.ctypes.data, self.signs.ctypes.data))
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.oq_rpbh_destroy(self.handle)
+            self.handle = None
+
+
+def oq_build_codebook(dim, bits):
+    return Codebook(dim, bits)
+
+
+def oq_make_rpbh(dim, block, seed):
+    return Rpbh(dim, block, seed)
+
+
+def oq_packed_bytes(rows, dim, bits):
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(lib().oq_packed_bytes(rows, dim, bits, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def _alloc_packed(rows, dim, bits, device):
+    import torch
+    total, pitch = oq_packed_bytes(rows, dim, bits)
+    return torch.empty((rows, pitch), dtype=torch.uint8, device=device)
+
+
+def oq_rotate_quantize_act(X, rot, cb_a, out_idx=None, out_norm=None, dbg_rotated=None):
+    """X: CUDA bf16 [N, d] (row stride = ldx).  Returns (packed uint8 [N, pitch], norm fp32 [N])."""
+    import torch
+    n, d = X.shape
+    if out_idx is None:
+        out_idx = _alloc_packed(n, d, cb_a.bits, X.device)
+    if out_norm is None:
+        out_norm = torch.empty(n, dtype=torch.float32, device=X.device)
+    _check(lib().oq_rotate_quantize_act(_ptr(X), n, d, X.stride(0) if n > 1 else d, rot.handle, cb_a.handle,
+                                        _ptr(out_idx), _ptr(out_norm), _ptr(dbg_rotated), _stream()))
+    return out_idx, out_norm
+
+
+def oq_quantize_weights(W, rot, cb_w, out_idx=None, out_norm=None, dbg_rotated=None):
+    """W: CUDA bf16 [m, d].  Returns (packed uint8 [m, pitch], row norms bf16 [m])."""
+    import torch
+    m, d = W.shape
+    if out_idx is None:
+        out_idx = _alloc_packed(m, d, cb_w.bits, W.device)
+    if out_norm is None:
+        out_norm = torch.empty(m, dtype=torch.bfloat16, device=W.device)
+    _check(lib().oq_quantize_weights(_ptr(W), m, d, W.stride(0) if m > 1 else d, rot.handle, cb_w.handle,
+                                     _ptr(out_idx), _ptr(out_norm), _ptr(dbg_rotated), _stream()))
+    return out_idx, out_norm
+
+
+def oq_qlinear(Xq_idx, Xq_norm, cb_a, Wq_idx, Wq_norm, cb_w, dim, out=None, out_dtype=None):
+    """Returns Y [N, m] (bf16 by default, fp32 when out_dtype is torch.float32)."""
+    import torch
+    n, m = Xq_idx.shape[0], Wq_idx.shape[0]
+    if out is None:
+        out = torch.empty((n, m), dtype=out_dtype or torch.bfloat16, device=Xq_idx.device)
+    ydt = OQ_F32 if out.dtype == torch.float32 else OQ_BF16
+    _check(lib().oq_qlinear(_ptr(Xq_idx), _ptr(Xq_norm), n, cb_a.handle, _ptr(Wq_idx), _ptr(Wq_norm), m,
+                            cb_w.handle, dim, _ptr(out), out.stride(0) if n > 1 else m, ydt, _stream()))
+    return out
+
+
+def oq_unpack_indices(idx, rows, dim, bits):
+    import torch
+    out = torch.empty((rows, dim), dtype=torch.uint8, device=idx.device)
+    _check(lib().oq_unpack_indices(_ptr(idx), rows, dim, bits, _ptr(out), _stream()))
+    return out
+
+
+def oq_device_status():
+    s = C.c_int(0)
+    code = lib().oq_device_status(C.byref(s))
+    if code not in (0, 5):
+        _check(code)
+    return s.value
+
+
+def oq_version():
+    return lib().oq_version().decode()

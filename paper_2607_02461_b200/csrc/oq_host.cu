@@ -1,0 +1,291 @@
+// Host side of liboq: error reporting, the two offline constructors (Lloyd-Max codebook, RPBH draw),
+// size queries and the device status word.
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <new>
+
+#include "oq_internal.h"
+
+namespace oq {
+
+static thread_local std::string g_last_error;
+
+int fail(int code, const std::string& msg) {
+  g_last_error = msg;
+  return code;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+  return fail(OQ_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Lloyd-Max on the sphere-coordinate marginal (Eq. 2-3).
+//
+// Unnormalised density g(t) = (1 - t^2)^((d-3)/2).  Cell mass by Gauss-Legendre quadrature on sub-cells
+// no wider than half a standard deviation (1/sqrt(d)); the unbounded-looking outer cell is cut 16
+// standard deviations above its lower edge, where g has fallen below 1e-55 of its peak.  Cell first
+// moment in closed form: int_a^b t g(t) dt = [(1-a^2)^p - (1-b^2)^p] / (d-1), p = (d-1)/2.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kGL = 16;  // 32-point rule, symmetric half stored
+// Abscissae / weights of the 32-point Gauss-Legendre rule on [-1, 1] are computed at start-up by
+// Newton iteration on the Legendre polynomial (no table to mistype).
+struct GL32 {
+  double x[2 * kGL], w[2 * kGL];
+  GL32() {
+    const int n = 2 * kGL;
+    for (int i = 0; i < n; ++i) {
+      double z = std::cos(M_PI * (i + 0.75) / (n + 0.5));
+      double pp = 1.0;
+      for (int it = 0; it < 100; ++it) {
+        double p1 = 1.0, p2 = 0.0;
+        for (int j = 0; j < n; ++j) {
+          double p3 = p2;
+          p2 = p1;
+          p1 = ((2.0 * j + 1.0) * z * p2 - j * p3) / (j + 1.0);
+        }
+        pp = n * (z * p1 - p2) / (z * z - 1.0);
+        double dz = p1 / pp;
+        z -= dz;
+        if (std::fabs(dz) < 1e-16) break;
+      }
+      x[i] = z;
+      w[i] = 2.0 / ((1.0 - z * z) * pp * pp);
+    }
+  }
+};
+const GL32& gl32() {
+  static GL32 g;
+  return g;
+}
+
+double cell_mass(double lo, double hi, int d) {
+  const double sigma = 1.0 / std::sqrt((double)d);
+  hi = std::fmin(hi, std::fmin(1.0, lo + 16.0 * sigma));
+  if (!(hi > lo)) return 0.0;
+  const double e = 0.5 * (d - 3);
+  int nsub = (int)std::ceil((hi - lo) / (0.5 * sigma));
+  if (nsub < 1) nsub = 1;
+  const GL32& q = gl32();
+  double total = 0.0;
+  const double wsub = (hi - lo) / nsub;
+  for (int s = 0; s < nsub; ++s) {
+    const double a = lo + s * wsub, half = 0.5 * wsub, mid = a + half;
+    double acc = 0.0;
+    for (int i = 0; i < 2 * kGL; ++i) {
+      const double t = mid + half * q.x[i];
+      const double u = 1.0 - t * t;
+      acc += q.w[i] * (u > 0.0 ? std::exp(e * std::log1p(-t * t)) : 0.0);
+    }
+    total += acc * half;
+  }
+  return total;
+}
+
+double cell_moment(double lo, double hi, int d) {
+  const double p = 0.5 * (d - 1);
+  auto prim = [&](double t) { return t < 1.0 ? std::exp(p * std::log1p(-t * t)) : 0.0; };
+  return (prim(lo) - prim(hi)) / (d - 1);
+}
+
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+CodebookParams codebook_params(const oq_codebook* cb) {
+  CodebookParams p;
+  const int L = 1 << cb->bits, M = L / 2;
+  for (int j = 0; j < 8; ++j) p.pos_bound[j] = std::numeric_limits<float>::infinity();
+  for (int j = 1; j < M; ++j) p.pos_bound[j - 1] = cb->boundaries_f32[M - 1 + j];
+  for (int j = 0; j < 16; ++j) p.level_bf16[j] = j < L ? cb->centroids_bf16[j] : 0;
+  p.bits = cb->bits;
+  return p;
+}
+
+static int* g_status_word[64] = {nullptr};
+
+int* device_status_word() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!g_status_word[dev]) {
+    int* p = nullptr;
+    if (cudaMalloc(&p, sizeof(int)) != cudaSuccess) return nullptr;
+    if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return nullptr;
+    g_status_word[dev] = p;
+  }
+  return g_status_word[dev];
+}
+
+int ensure_device_tables(const oq_rpbh* rc) {
+  oq_rpbh* r = const_cast<oq_rpbh*>(rc);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (r->d_gather && r->device == dev) return OQ_OK;
+  if (r->d_gather) return fail(OQ_ERR_INVALID_ARG, "rpbh handle was first used on another device");
+  std::vector<uint32_t> g(r->dim);
+  for (int k = 0; k < r->dim; ++k) g[k] = (uint32_t)r->perm[k] | (r->signs[k] < 0 ? 0x80000000u : 0u);
+  e = cudaMalloc(&r->d_gather, sizeof(uint32_t) * r->dim);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
+  e = cudaMemcpy(r->d_gather, g.data(), sizeof(uint32_t) * r->dim, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
+  r->device = dev;
+  return OQ_OK;
+}
+
+}  // namespace oq
+
+using namespace oq;
+
+extern "C" {
+
+const char* oq_last_error(void) { return g_last_error.c_str(); }
+const char* oq_version(void) { return "liboq 0.1 (sm_100a)"; }
+
+int oq_build_codebook(int dim, int bits, oq_codebook** out) {
+  if (!out) return fail(OQ_ERR_INVALID_ARG, "oq_build_codebook: out is NULL");
+  *out = nullptr;
+  if (dim < 16) return fail(OQ_ERR_UNSUPPORTED, "oq_build_codebook: dim must be >= 16");
+  if (bits < 1 || bits > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_build_codebook: bits must be in 1..4");
+  const int L = 1 << bits, M = L / 2;
+  const double sigma = 1.0 / std::sqrt((double)dim);
+  std::vector<double> c(M), edge(M + 1);
+  for (int j = 0; j < M; ++j) c[j] = std::fmin(3.0 * sigma, 1.0) * (2 * j + 1) / (2.0 * M);
+  // Plain Lloyd iteration on the positive half (the density is even).  It contracts linearly (ratio
+  // about 0.965 at 4 bits), so it runs until the step is at rounding level, with an iteration cap.
+  for (int it = 0; it < 20000; ++it) {
+    edge[0] = 0.0;
+    for (int j = 1; j < M; ++j) edge[j] = 0.5 * (c[j - 1] + c[j]);
+    edge[M] = 1.0;
+    double step = 0.0;
+    for (int j = 0; j < M; ++j) {
+      const double nc = cell_moment(edge[j], edge[j + 1], dim) / cell_mass(edge[j], edge[j + 1], dim);
+      step = std::fmax(step, std::fabs(nc - c[j]));
+      c[j] = nc;
+    }
+    if (step <= 2e-17 * c[M - 1]) break;
+  }
+  oq_codebook* cb = new (std::nothrow) oq_codebook;
+  if (!cb) return fail(OQ_ERR_NOMEM, "oq_build_codebook: out of host memory");
+  cb->dim = dim;
+  cb->bits = bits;
+  cb->centroids.resize(L);
+  cb->boundaries.resize(L - 1);
+  for (int j = 0; j < M; ++j) {
+    cb->centroids[M + j] = c[j];
+    cb->centroids[M - 1 - j] = -c[j];
+  }
+  for (int j = 0; j < L - 1; ++j) cb->boundaries[j] = 0.5 * (cb->centroids[j] + cb->centroids[j + 1]);
+  cb->boundaries[M - 1] = 0.0;
+  cb->boundaries_f32.resize(L - 1);
+  cb->centroids_bf16.resize(L);
+  for (int j = 0; j < L - 1; ++j) cb->boundaries_f32[j] = (float)cb->boundaries[j];
+  for (int j = 0; j < L; ++j) cb->centroids_bf16[j] = f32_to_bf16_rne((float)cb->centroids[j]);
+  *out = cb;
+  return OQ_OK;
+}
+
+int oq_codebook_get(const oq_codebook* cb, double* centroids, double* boundaries, float* boundaries_f32,
+                    uint16_t* centroids_bf16) {
+  if (!cb) return fail(OQ_ERR_INVALID_ARG, "oq_codebook_get: handle is NULL");
+  const int L = 1 << cb->bits;
+  if (centroids) std::memcpy(centroids, cb->centroids.data(), sizeof(double) * L);
+  if (boundaries) std::memcpy(boundaries, cb->boundaries.data(), sizeof(double) * (L - 1));
+  if (boundaries_f32) std::memcpy(boundaries_f32, cb->boundaries_f32.data(), sizeof(float) * (L - 1));
+  if (centroids_bf16) std::memcpy(centroids_bf16, cb->centroids_bf16.data(), sizeof(uint16_t) * L);
+  return OQ_OK;
+}
+int oq_codebook_dim(const oq_codebook* cb) { return cb ? cb->dim : 0; }
+int oq_codebook_bits(const oq_codebook* cb) { return cb ? cb->bits : 0; }
+void oq_codebook_destroy(oq_codebook* cb) { delete cb; }
+
+int oq_make_rpbh(int dim, int block, uint64_t seed, oq_rpbh** out) {
+  if (!out) return fail(OQ_ERR_INVALID_ARG, "oq_make_rpbh: out is NULL");
+  *out = nullptr;
+  if (dim <= 0 || dim >= 65536) return fail(OQ_ERR_UNSUPPORTED, "oq_make_rpbh: dim must be in 1..65535");
+  if (block <= 0 || (block & (block - 1)) || dim % block)
+    return fail(OQ_ERR_INVALID_ARG, "oq_make_rpbh: block must be a power of two that divides dim");
+  oq_rpbh* r = new (std::nothrow) oq_rpbh;
+  if (!r) return fail(OQ_ERR_NOMEM, "oq_make_rpbh: out of host memory");
+  r->dim = dim;
+  r->block = block;
+  r->seed = seed;
+  uint64_t state = seed ^ ((uint64_t)(uint32_t)dim << 32) ^ (uint64_t)block;
+  auto next = [&state]() {
+    state += 0x9E3779B97F4A7C15ull;
+    uint64_t z = state;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+  };
+  r->perm.resize(dim);
+  for (int i = 0; i < dim; ++i) r->perm[i] = i;
+  for (int i = dim - 1; i >= 1; --i) {
+    const uint64_t n = (uint64_t)i + 1;
+    const uint64_t thr = (0 - n) % n;  // (2^64 - n) mod n
+    uint64_t v;
+    do v = next();
+    while (v < thr);
+    const int j = (int)(v % n);
+    const int32_t t = r->perm[i];
+    r->perm[i] = r->perm[j];
+    r->perm[j] = t;
+  }
+  r->signs.resize(dim);
+  for (int base = 0; base < dim; base += 64) {
+    const uint64_t word = next();
+    for (int b = 0; b < 64 && base + b < dim; ++b) r->signs[base + b] = ((word >> b) & 1) ? -1 : 1;
+  }
+  *out = r;
+  return OQ_OK;
+}
+
+int oq_rpbh_get(const oq_rpbh* r, int32_t* perm, int8_t* signs) {
+  if (!r) return fail(OQ_ERR_INVALID_ARG, "oq_rpbh_get: handle is NULL");
+  if (perm) std::memcpy(perm, r->perm.data(), sizeof(int32_t) * r->dim);
+  if (signs) std::memcpy(signs, r->signs.data(), r->dim);
+  return OQ_OK;
+}
+int oq_rpbh_dim(const oq_rpbh* r) { return r ? r->dim : 0; }
+int oq_rpbh_block(const oq_rpbh* r) { return r ? r->block : 0; }
+void oq_rpbh_destroy(oq_rpbh* r) {
+  if (!r) return;
+  if (r->d_gather) cudaFree(r->d_gather);
+  delete r;
+}
+
+int oq_packed_bytes(int rows, int dim, int bits, size_t* idx_bytes, size_t* row_pitch_bytes) {
+  if (rows < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, "oq_packed_bytes: bad sizes");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, "oq_packed_bytes: dim must be a multiple of 128");
+  if (bits < 2 || bits > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_packed_bytes: bits must be 2, 3 or 4");
+  const size_t pitch = (size_t)dim / 8 * bits;  // dim % 128 == 0 makes this a multiple of 16
+  if (row_pitch_bytes) *row_pitch_bytes = pitch;
+  if (idx_bytes) *idx_bytes = pitch * (size_t)rows;
+  return OQ_OK;
+}
+
+int oq_device_status(int* status) {
+  if (!status) return fail(OQ_ERR_INVALID_ARG, "oq_device_status: status is NULL");
+  *status = 0;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
+  int* w = device_status_word();
+  if (!w) return fail(OQ_ERR_CUDA, "oq_device_status: no status word (no usable device?)");
+  e = cudaMemcpy(status, w, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+  if (*status != 0) {
+    cudaMemset(w, 0, sizeof(int));
+    return fail(OQ_ERR_DEVICE_TIMEOUT, "a bounded device-side wait gave up; status code " + std::to_string(*status));
+  }
+  return OQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,187 @@
+// Fused per-row pass: norm -> RPBH rotation -> nearest Lloyd-Max level -> bit-pack
+// (Eq. 7-8 for activations, Eq. 4-6 for weight rows).
+#include <cuda_bf16.h>
+
+#include "oq_internal.h"
+#include "oq_packing.cuh"
+
+namespace oq {
+
+// -----------------------------------------------------------------------------------------------------
+// General kernel: any power-of-two block size up to dim.  One CTA per row (grid-stride over rows), the
+// row lives in shared memory as fp32 and the Walsh-Hadamard butterflies run there.
+// -----------------------------------------------------------------------------------------------------
+template <bool kBf16Norm>
+__global__ void __launch_bounds__(256)
+rq_general_kernel(const __nv_bfloat16* __restrict__ X, int rows, int dim, int ldx, int block,
+                  const uint32_t* __restrict__ gather, CodebookParams cb, uint32_t* __restrict__ out_idx,
+                  int pitch_words, void* __restrict__ out_norm, float* __restrict__ dbg) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* z = reinterpret_cast<float*>(smem_raw);
+  uint8_t* lvl = reinterpret_cast<uint8_t*>(z + dim);
+  __shared__ float red[8];
+  __shared__ float s_norm;
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int M = (1 << cb.bits) >> 1;
+  const float inv_sqrt_h = rsqrtf((float)block);
+
+  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    const __nv_bfloat16* x = X + (size_t)row * ldx;
+    float ss = 0.f;
+    for (int k = tid; k < dim; k += nthr) {
+      const uint32_t g = gather[k];
+      float v = __bfloat162float(x[g & 0xFFFFu]);
+      ss = fmaf(v, v, ss);
+      z[k] = (g >> 31) ? -v : v;
+    }
+    for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();
+    if (tid == 0) {
+      float t = 0.f;
+      for (int w = 0; w < (nthr >> 5); ++w) t += red[w];
+      s_norm = sqrtf(t);
+    }
+    for (int len = 1; len < block; len <<= 1) {
+      __syncthreads();
+      for (int p = tid; p < dim / 2; p += nthr) {
+        const int i = ((p / len) * 2 * len) + (p % len);
+        const float a = z[i], b = z[i + len];
+        z[i] = a + b;
+        z[i + len] = a - b;
+      }
+    }
+    __syncthreads();
+    const float s = s_norm;
+    if (tid == 0) {
+      if (kBf16Norm) reinterpret_cast<__nv_bfloat16*>(out_norm)[row] = __float2bfloat16_rn(s);
+      else reinterpret_cast<float*>(out_norm)[row] = s;
+    }
+    // thresholds for the un-normalised butterfly output: beta_j * sqrt(h) * (s + eps)
+    const float scale = (s + 1e-10f) * sqrtf((float)block);
+    for (int k = tid; k < dim; k += nthr) {
+      const float v = z[k];
+      const float a = fabsf(v);
+      int mag = 0;
+      for (int j = 0; j < M - 1; ++j) mag += (a > cb.pos_bound[j] * scale) ? 1 : 0;
+      lvl[k] = (uint8_t)((v > 0.f) ? M + mag : M - 1 - mag);
+      if (dbg) dbg[(size_t)row * dim + k] = v * inv_sqrt_h;
+    }
+    __syncthreads();
+    uint32_t* orow = out_idx + (size_t)row * pitch_words;
+    // one thread per 32 coordinates builds that group's words
+    for (int g = tid; g < dim / 32; g += nthr) {
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      const int w0 = field_pos(cb.bits, 32 * g).mag_word < field_pos(cb.bits, 32 * g).sign_word
+                         ? field_pos(cb.bits, 32 * g).mag_word : field_pos(cb.bits, 32 * g).sign_word;
+      for (int kp = 0; kp < 32; ++kp) {
+        const int idx = lvl[32 * g + kp];
+        const int sgn = idx < M;
+        const uint32_t mag = sgn ? M - 1 - idx : idx - M;
+        const FieldPos p = field_pos(cb.bits, 32 * g + kp);
+        w[p.mag_word - w0] |= mag << p.mag_shift;
+        w[p.sign_word - w0] |= (uint32_t)sgn << p.sign_bit;
+      }
+      for (int i = 0; i < cb.bits; ++i) orow[w0 + i] = w[i];
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void unpack_kernel(const uint32_t* __restrict__ idx, int rows, int dim, int bits, int pitch_words,
+                              uint8_t* __restrict__ out) {
+  const size_t total = (size_t)rows * dim;
+  const int M = (1 << bits) >> 1;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / dim), k = (int)(i % dim);
+    const FieldPos p = field_pos(bits, k);
+    const uint32_t* r = idx + (size_t)row * pitch_words;
+    const int mag = (r[p.mag_word] >> p.mag_shift) & (M - 1);
+    const int sgn = (r[p.sign_word] >> p.sign_bit) & 1;
+    out[i] = (uint8_t)(sgn ? M - 1 - mag : M + mag);
+  }
+}
+
+static int check_common(const char* fn, const void* X, int rows, int dim, int ld, const oq_rpbh* rot,
+                        const oq_codebook* cb, const void* out_idx, const void* out_norm) {
+  if (!rot || !cb) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": NULL handle");
+  if (rows < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": bad sizes");
+  if (rot->dim != dim || cb->dim != dim)
+    return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": dim differs from the rotation's or the codebook's");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, std::string(fn) + ": dim must be a multiple of 128");
+  if (cb->bits < 2 || cb->bits > 4) return fail(OQ_ERR_UNSUPPORTED, std::string(fn) + ": bits must be 2, 3 or 4");
+  if (rows == 0) return OQ_OK;
+  if (!X || !out_idx || !out_norm) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": NULL buffer");
+  if (ld < dim) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": leading dimension smaller than dim");
+  if (ld % 8 || !aligned16(X) || !aligned16(out_idx))
+    return fail(OQ_ERR_ALIGNMENT, std::string(fn) + ": pointers must be 16-byte aligned and ld a multiple of 8");
+  return OQ_OK;
+}
+
+template <bool kBf16Norm>
+static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, const oq_rpbh* rot,
+                     const oq_codebook* cb, void* out_idx, void* out_norm, float* dbg, void* stream) {
+  int rc = check_common(fn, X, rows, dim, ld, rot, cb, out_idx, out_norm);
+  if (rc != OQ_OK || rows == 0) return rc;
+  rc = ensure_device_tables(rot);
+  if (rc != OQ_OK) return rc;
+  const CodebookParams cp = codebook_params(cb);
+  const int pitch_words = dim / 32 * cb->bits;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  const size_t smem = (size_t)dim * 5;
+  auto kern = rq_general_kernel<kBf16Norm>;
+  if (smem > 48 * 1024) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute");
+  }
+  int per_sm = 1;
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, smem);
+  if (per_sm < 1) per_sm = 1;
+  int grid = sms * per_sm;
+  if (grid > rows) grid = rows;
+  kern<<<grid, 256, smem, st>>>(reinterpret_cast<const __nv_bfloat16*>(X), rows, dim, ld, rot->block, rot->d_gather,
+                                cp, reinterpret_cast<uint32_t*>(out_idx), pitch_words, out_norm, dbg);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, fn);
+  return OQ_OK;
+}
+
+}  // namespace oq
+
+using namespace oq;
+
+extern "C" {
+
+int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                           const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated,
+                           void* stream) {
+  return launch_rq<false>("oq_rotate_quantize_act", X_bf16, n_tokens, dim, ldx, rot, cb_a, Xq_idx, Xq_norm,
+                          dbg_rotated, stream);
+}
+
+int oq_quantize_weights(const void* W_bf16, int m, int dim, int ldw, const oq_rpbh* rot, const oq_codebook* cb_w,
+                        void* Wq_idx, void* Wq_norm_bf16, void* dbg_rotated, void* stream) {
+  return launch_rq<true>("oq_quantize_weights", W_bf16, m, dim, ldw, rot, cb_w, Wq_idx, Wq_norm_bf16,
+                         reinterpret_cast<float*>(dbg_rotated), stream);
+}
+
+int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream) {
+  if (rows < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, "oq_unpack_indices: bad sizes");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, "oq_unpack_indices: dim must be a multiple of 128");
+  if (bits < 2 || bits > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_unpack_indices: bits must be 2, 3 or 4");
+  if (rows == 0) return OQ_OK;
+  if (!idx || !out) return fail(OQ_ERR_INVALID_ARG, "oq_unpack_indices: NULL buffer");
+  const size_t total = (size_t)rows * dim;
+  int grid = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+  unpack_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<const uint32_t*>(idx), rows, dim, bits, dim / 32 * bits, out);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "oq_unpack_indices");
+  return OQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+"""GPU parity of oq_rotate_quantize_act / oq_quantize_weights against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+
+from oracle import bf16 as obf
+from oracle import codebook as ocb
+from oracle import quantize as oq
+from oracle import rpbh as orp
+from paper_2607_02461_b200 import binding as B
+from paper_2607_02461_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+ROT_TOL = 1e-5      # rotated activations: relative to the token's largest coordinate / Frobenius
+BAND = 1e-5         # a level flip is allowed only within this (times the token's largest |t|) of a boundary
+
+
+def _dev(bits_u16):
+    import torch
+    return torch.from_numpy(bits_u16.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def check_rows(xb, block, seed, bits, weights=False, rows=None):
+    """Runs the GPU pass on xb (uint16 bf16 bits [N, d]) and compares with the oracle on `rows`."""
+    import torch
+    n, d = xb.shape
+    rot, cb = B.oq_make_rpbh(d, block, seed), B.oq_build_codebook(d, bits)
+    X = _dev(xb)
+    dbg = torch.full((n, d), float("nan"), dtype=torch.float32, device="cuda")
+    fn = B.oq_quantize_weights if weights else B.oq_rotate_quantize_act
+    idx_p, norm = fn(X, rot, cb, dbg_rotated=dbg)
+    idx = B.oq_unpack_indices(idx_p, n, d, bits).cpu().numpy()
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    sel = np.arange(n) if rows is None else np.asarray(rows)
+    perm, signs = orp.make_rpbh(d, block, seed)
+    ocbk = ocb.lloyd_max(d, bits)
+    ref = (oq.quantize_weight_rows if weights else oq.quantize_rows)(xb[sel], block, perm, signs, ocbk.boundaries)
+    z_gpu = dbg.cpu().numpy()[sel].astype(np.float64)
+    z_ref = ref["rotated"]
+    tok_max = np.abs(z_ref).max(axis=1)
+    assert np.all(np.abs(z_gpu - z_ref).max(axis=1) <= ROT_TOL * tok_max + 1e-300)
+    assert np.linalg.norm(z_gpu - z_ref) <= ROT_TOL * np.linalg.norm(z_ref) + 1e-300
+    if weights:
+        got = norm.view(torch.int16).cpu().numpy().view(np.uint16)[sel]
+        want = ref["norm_bf16_bits"]
+        off = got.astype(np.int32) - want.astype(np.int32)
+        assert np.abs(off).max() <= 1                         # fp32 vs fp64 norm may straddle a bf16 rounding edge
+        assert (off != 0).mean() <= 0.01
+    else:
+        got = norm.cpu().numpy()[sel].astype(np.float64)
+        assert np.all(np.abs(got - ref["norm"]) <= 1e-6 * ref["norm"])
+    # level indices: bit-exact except adjacent-bin flips inside the band around a boundary
+    gi, ri = idx[sel].astype(np.int32), ref["idx"].astype(np.int32)
+    flips = np.argwhere(gi != ri)
+    tmax = np.abs(ref["unit"]).max(axis=1)
+    for r, k in flips:
+        assert abs(gi[r, k] - ri[r, k]) == 1
+        beta = ocbk.boundaries[min(gi[r, k], ri[r, k])]
+        assert abs(ref["unit"][r, k] - beta) <= BAND * tmax[r]
+    return len(flips) / gi.size
+
+
+@pytest.mark.parametrize("bits", [4, 3, 2])
+@pytest.mark.parametrize("d,block", [(1024, 128), (384, 64), (768, 256), (1024, 1024), (128, 8)])
+def test_activation_rows_match_oracle(d, block, bits):
+    xb = synth.activations(67, d, seed=1000 + bits)        # 67 rows: ragged against any row tiling
+    rate = check_rows(xb, block, 0, bits)
+    assert rate <= 1e-4
+
+
+def test_config1_single_linear_activation_side():
+    xb = synth.activations(256, 1024, seed=1000)
+    assert check_rows(xb, 128, 0, 4) <= 1e-5
+
+
+@pytest.mark.parametrize("bits", [4, 3, 2])
+def test_weight_rows_match_oracle(bits):
+    wb = synth.weights(200, 1024, seed=2000)
+    wb[17, :] = 0
+    assert check_rows(wb, 128, 0, bits, weights=True) <= 1e-4
+
+
+def test_degenerate_tokens_and_strided_input():
+    import torch
+    d = 512
+    x = np.zeros((5, d), np.float32)
+    x[1, 100] = 30000.0
+    x[2, :] = 1.5
+    x[3, ::2] = -2.0 ** -120          # tiny values: squares underflow in fp32
+    x[4, :] = np.random.default_rng(0).standard_normal(d) * 1e4
+    xb = synth.to_bf16_bits(x)
+    assert check_rows(xb, 128, 3, 4, rows=[0, 1, 2, 4]) <= 2e-3   # exact zeros sit on the middle boundary (ties)
+    rot, cb = B.oq_make_rpbh(d, 128, 3), B.oq_build_codebook(d, 4)
+    # leading dimension larger than dim
+    wide = torch.zeros((5, d + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :d] = _dev(xb)
+    a_idx, a_norm = B.oq_rotate_quantize_act(wide[:, :d], rot, cb)
+    b_idx, b_norm = B.oq_rotate_quantize_act(_dev(xb), rot, cb)
+    assert torch.equal(a_idx, b_idx) and torch.equal(a_norm, b_norm)
+    assert a_norm[0].item() == 0.0
+    assert torch.all(B.oq_unpack_indices(a_idx, 5, d, 4)[0] == 7)
+
+
+def test_empty_and_bad_arguments():
+    import torch
+    d = 256
+    rot, cb = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, 4)
+    X = torch.zeros((0, d), dtype=torch.bfloat16, device="cuda")
+    idx, nrm = B.oq_rotate_quantize_act(X, rot, cb)
+    assert idx.shape[0] == 0 and nrm.numel() == 0
+    with pytest.raises(B.OqError) as e:
+        B.oq_rotate_quantize_act(torch.zeros((4, 384), dtype=torch.bfloat16, device="cuda"), rot, cb)
+    assert e.value.code == 1
+    X = torch.zeros((4, d + 8), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.OqError) as e:
+        B.oq_rotate_quantize_act(X.view(-1)[1:1 + 4 * d].view(4, d), rot, cb)
+    assert e.value.code == 3
+
+
+def test_results_are_deterministic():
+    import torch
+    xb = synth.activations(300, 3072, seed=1001)
+    rot, cb = B.oq_make_rpbh(3072, 128, 0), B.oq_build_codebook(3072, 4)
+    X = _dev(xb)
+    a = B.oq_rotate_quantize_act(X, rot, cb)
+    b = B.oq_rotate_quantize_act(X, rot, cb)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
