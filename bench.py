@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the OrbitQuant quantized-linear hot path on B200.
+
+One STEP = the whole online path of the four linear layers of a FLUX.1-dev-shaped double-stream block
+at W4A4 on 4608 tokens: for every layer, fused rotate+quantize of its activations (norm -> RPBH ->
+Lloyd-Max level -> pack) followed by the codebook-decode GEMM.  Weights are quantized offline (not timed).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload flux_w4a4]
+
+Prints ONE JSON line (rank 0).  `value` = effective TFLOP/s of the whole step (2*N*m*d summed over the
+layers, divided by the device time of the step, rotate+quantize included), aggregated over ranks
+(token-sharded replicas, no collective).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_02461_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (tokens, layers, bits_w, bits_a, block)
+    "flux_w4a4": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 4, 4, 128),
+    "flux_w3a3": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 3, 3, 128),
+    "flux_w2a4": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 2, 4, 128),
+    "wan_w4a4": (synth.WAN_TOKENS, synth.WAN_LAYERS, 4, 4, 128),
+    "single_w4a4": (256, [("linear", 1024, 1024)], 4, 4, 128),
+}
+CONFIG_INDEX = {"single_w4a4": 0, "flux_w4a4": 1, "flux_w3a3": 1, "flux_w2a4": 2, "wan_w4a4": 3}
+METRIC = "qlinear effective TFLOP/s (whole step: rotate+quantize and codebook GEMM)"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops"],
+                "bf16_tflops_sustained": j.get("bf16_tflops_sustained", j["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def rq_bytes(n, d, bits):
+    return 2 * n * d + n * d * bits // 8 + 4 * n          # bf16 row in, packed indices + fp32 norm out
+
+
+# ----------------------------------------------------------------------------------------------------------
+# CPU oracle arm (also the cpu_baseline of the main arm)
+# ----------------------------------------------------------------------------------------------------------
+def oracle_sample(workload, sample_tokens=512, sample_rows=1024):
+    """Builds the oracle's inputs for a bounded sample of the workload; returns a closure running one
+    sample step (rotate+quantize of `sample_tokens` tokens and the fp64 product against `sample_rows`
+    weight rows, for every layer) and the flops of that sample."""
+    from oracle import bf16 as obf
+    from oracle import codebook as ocb
+    from oracle import qlinear as oql
+    from oracle import quantize as oq
+    from oracle import rpbh as orp
+    tokens, layers, bw, ba, block = WORKLOADS[workload]
+    ci = CONFIG_INDEX[workload]
+    nt = min(tokens, sample_tokens)
+    prep = []
+    flops = 0
+    for li, (name, d, m) in enumerate(layers):
+        mr = min(m, sample_rows)
+        perm, signs = orp.make_rpbh(d, block, 0)
+        ca, cw = ocb.lloyd_max(d, ba), ocb.lloyd_max(d, bw)
+        xb = synth.activations(nt, d, 1000 + ci)
+        wb = synth.weights(mr, d, 2000 + 10 * ci + li)
+        qw = oq.quantize_weight_rows(wb, block, perm, signs, cw.boundaries)        # offline, not timed
+        r = obf.bf16_bits_to_f64(qw["norm_bf16_bits"])
+        prep.append((xb, block, perm, signs, ca, cw, qw["idx"], r))
+        flops += 2 * nt * mr * d
+
+    def step():
+        for xb, block_, perm, signs, ca, cw, iw, r in prep:
+            qa = oq.quantize_rows(xb, block_, perm, signs, ca.boundaries)
+            oql.qlinear(qa["idx"], qa["norm"].astype(np.float32), ca.centroids_decoded, iw, r, cw.centroids_decoded)
+
+    desc = f"{nt} of {tokens} tokens x first {sample_rows} weight rows of each of {len(layers)} layers ({workload})"
+    return step, flops, desc
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    step, flops, desc = oracle_sample(args.workload)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = flops / dt / 1e12
+    cores = min(blas_threads(), len(os.sched_getaffinity(0)))
+    tokens, layers, bw, ba, block = WORKLOADS[args.workload]
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "tokens": tokens, "layers": [l[0] for l in layers],
+                   "bits_w": bw, "bits_a": ba, "rpbh_block": block, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, reasons = [], set()
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                out["sm_max_mhz"] = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_02461_b200 import binding as B
+    from paper_2607_02461_b200 import build as oqbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    oqbuild.build()
+    B.lib()
+
+    tokens, layers, bw, ba, block = WORKLOADS[args.workload]
+    ci = CONFIG_INDEX[args.workload]
+    dev = torch.device("cuda", local)
+    to_dev = lambda b: torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    # ---- offline: codebooks, rotation, weight quantization (not timed) ----
+    L = []
+    for li, (name, d, m) in enumerate(layers):
+        rot = B.oq_make_rpbh(d, block, 0)
+        cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
+        xb = synth.activations(tokens, d, 1000 + ci + 100 * rank)           # every rank has its own tokens
+        wb = synth.weights(m, d, 2000 + 10 * ci + li)
+        Xh = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        X = Xh.to(dev)
+        wq, wr = B.oq_quantize_weights(to_dev(wb), rot, cbw)
+        xq = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device=dev)
+        xs = torch.empty(tokens, dtype=torch.float32, device=dev)
+        Y = torch.empty((tokens, m), dtype=torch.bfloat16, device=dev)
+        Yh = torch.empty((tokens, m), dtype=torch.bfloat16).pin_memory()
+        ws = torch.empty(B.oq_forward_workspace_bytes(tokens, d, m, ba), dtype=torch.uint8, device=dev)
+        L.append(dict(name=name, d=d, m=m, rot=rot, cba=cba, cbw=cbw, X=X, Xh=Xh, wq=wq, wr=wr, xq=xq, xs=xs, Y=Y,
+                      Yh=Yh, ws=ws))
+        del wb, xb
+    torch.cuda.synchronize()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)           # > L2 (126 MB)
+
+    def step(events=None):
+        for l in L:
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+            B.oq_rotate_quantize_act(l["X"], l["rot"], l["cba"], out_idx=l["xq"], out_norm=l["xs"])
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+            B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+        if events is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    all_events = []
+    t_wall = time.perf_counter()
+    for _ in range(args.steps):
+        flush.zero_()                                  # L2 flush between steps (outside the event-timed span)
+        ev = []
+        step(ev)
+        all_events.append(ev)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop() if sampler else None
+    status = B.oq_device_status()
+
+    step_ms = [ev[0].elapsed_time(ev[-1]) for ev in all_events]
+    rq_ms = np.zeros(len(L)); gemm_ms = np.zeros(len(L))
+    for ev in all_events:
+        for i in range(len(L)):
+            rq_ms[i] += ev[2 * i].elapsed_time(ev[2 * i + 1])
+            gemm_ms[i] += ev[2 * i + 1].elapsed_time(ev[2 * i + 2])
+    rq_ms /= args.steps; gemm_ms /= args.steps
+    total_ms = float(np.sum(step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    flops_step = sum(2 * tokens * l["m"] * l["d"] for l in L)
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point: H2D of every layer's tokens and D2H of every Y ----
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        for l in L:
+            B.oq_linear_forward_host(l["Xh"], l["rot"], l["cba"], l["wq"], l["wr"], l["cbw"], l["Yh"], l["ws"])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        for l in L:
+            B.oq_linear_forward_host(l["Xh"], l["rot"], l["cba"], l["wq"], l["wr"], l["cbw"], l["Yh"], l["ws"])
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(tokens * l["d"] * 2 for l in L)
+    d2h = sum(tokens * l["m"] * 2 for l in L)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    pk = peaks()
+    gemm_tf = sum(2 * tokens * l["m"] * l["d"] for l in L) / (float(np.sum(gemm_ms)) * 1e-3) / 1e12
+    rq_b = sum(rq_bytes(tokens, l["d"], ba) for l in L)
+    rq_gbs = rq_b / (float(np.sum(rq_ms)) * 1e-3) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        traffic = json.load(open(tpath)).get(args.workload, {})
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "tokens_per_gpu": tokens,
+                   "layers": [f"{l['name']} {l['d']}->{l['m']}" for l in L], "bits_w": bw, "bits_a": ba,
+                   "rpbh_block": block, "parallelism": f"token-sharded replicas x{world}, no collective",
+                   "l2": "256 MiB buffer written between steps, outside the event-timed spans"},
+        "roofline": {"bound": "tensor", "kernel": "qlinear_kernel", "achieved": gemm_tf,
+                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / pk["bf16_tflops"],
+                     "traffic": (traffic or {}).get("qlinear_bytes_per_step"),
+                     "peak_source": f"{pk['source']} burst (sustained {pk['bf16_tflops_sustained']})",
+                     "frac_of_nominal_2250": gemm_tf / 2250.0,
+                     "per_layer_tflops": {l["name"]: 2 * tokens * l["m"] * l["d"] / (gemm_ms[i] * 1e-3) / 1e12
+                                          for i, l in enumerate(L)}},
+        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
+                                     "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
+                                     "traffic": (traffic or {}).get("rq_bytes_per_step"),
+                                     "algorithmic_bytes_per_step": rq_b, "frac_of_nominal_8000": rq_gbs / 8000.0,
+                                     "per_layer_gbs": {l["name"]: rq_bytes(tokens, l["d"], ba) / (rq_ms[i] * 1e-3) / 1e9
+                                                       for i, l in enumerate(L)}},
+        "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": 2 * len(L) * args.steps,
+        "clocks": clocks, "device_status": status, "wall_s_timed_region": t_wall,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        stepf, flops, desc = oracle_sample(args.workload)
+        stepf()
+        t0 = time.perf_counter(); reps = 0
+        while reps < 3 or (time.perf_counter() - t0 < 10 and reps < 50):
+            stepf(); reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        out["cpu_baseline"] = {"value": flops / dt / 1e12, "unit": "TFLOP/s",
+                               "cores": min(blas_threads(), len(os.sched_getaffinity(0))), "kind": "oracle",
+                               "sample": desc + f", {reps} repetitions"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="flux_w4a4", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -124,6 +124,20 @@ int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_
                const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim,
                void* Y, int ldy, int y_dtype, void* stream);
 
+/* Whole online layer from HOST memory (Algorithm 1 "Online" followed by the product of Sec. 4.3):
+ * copies X (host, bf16 [n_tokens][dim], dense; pinned memory makes the copy asynchronous) to the device,
+ * runs oq_rotate_quantize_act and oq_qlinear, and copies Y (bf16 [n_tokens][m], dense) back to
+ * Y_host_bf16, all on `stream`.  Wq_idx / Wq_norm_bf16 are device buffers from oq_quantize_weights.
+ * `workspace` is a caller-owned device buffer of at least oq_forward_workspace_bytes() bytes (16-byte
+ * aligned); it holds X, the packed activations, the norms and Y while the call is in flight.
+ * The call returns after enqueueing; synchronise the stream before reading Y_host_bf16.
+ * Errors: as the two calls it wraps, OQ_ERR_NOMEM when the workspace is too small. */
+int oq_forward_workspace_bytes(int n_tokens, int dim, int m, int bits_a, size_t* bytes);
+int oq_linear_forward_host(const void* X_host_bf16, int n_tokens, int dim, const oq_rpbh* rot,
+                           const oq_codebook* cb_a, const void* Wq_idx, const void* Wq_norm_bf16, int m,
+                           const oq_codebook* cb_w, void* Y_host_bf16, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* Test helper: expand packed indices to one byte per coordinate, out dev [rows][dim] uint8, logical level
  * numbers in rotated-coordinate order. */
 int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream);

@@ -44,6 +44,8 @@ def lib():
             "oq_quantize_weights": (i, [vp, i, i, i, vp, vp, vp, vp, vp, vp]),
             "oq_qlinear": (i, [vp, vp, i, vp, vp, vp, i, vp, i, vp, i, i, vp]),
             "oq_unpack_indices": (i, [vp, i, i, i, vp, vp]),
+            "oq_forward_workspace_bytes": (i, [i, i, i, i, C.POINTER(sz)]),
+            "oq_linear_forward_host": (i, [vp, i, i, vp, vp, vp, vp, i, vp, vp, vp, sz, vp]),
             "oq_device_status": (i, [C.POINTER(i)]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
@@ -163,6 +165,21 @@ def oq_qlinear(Xq_idx, Xq_norm, cb_a, Wq_idx, Wq_norm, cb_w, dim, out=None, out_
     _check(lib().oq_qlinear(_ptr(Xq_idx), _ptr(Xq_norm), n, cb_a.handle, _ptr(Wq_idx), _ptr(Wq_norm), m,
                             cb_w.handle, dim, _ptr(out), out.stride(0) if n > 1 else m, ydt, _stream()))
     return out
+
+
+def oq_forward_workspace_bytes(n_tokens, dim, m, bits_a):
+    b = C.c_size_t()
+    _check(lib().oq_forward_workspace_bytes(n_tokens, dim, m, bits_a, C.byref(b)))
+    return b.value
+
+
+def oq_linear_forward_host(X_host, rot, cb_a, Wq_idx, Wq_norm, cb_w, Y_host, workspace):
+    """X_host / Y_host: CPU bf16 tensors (pinned for asynchronous copies); workspace: CUDA uint8 tensor."""
+    n, d = X_host.shape
+    m = Wq_idx.shape[0]
+    _check(lib().oq_linear_forward_host(_ptr(X_host), n, d, rot.handle, cb_a.handle, _ptr(Wq_idx), _ptr(Wq_norm), m,
+                                        cb_w.handle, _ptr(Y_host), _ptr(workspace), workspace.numel(), _stream()))
+    return Y_host
 
 
 def oq_unpack_indices(idx, rows, dim, bits):

@@ -49,10 +49,11 @@ def run_case(n, m, d, ba, bw, block=128, seed=0, xseed=1000, wseed=2000, end_to_
     g16 = y16.float().cpu().numpy().astype(np.float64)
     assert _rel(g32, ref) <= TOL_F32
     assert _rel(g16, ref) <= TOL_BF16
-    # bf16 output must be the fp32 result rounded once: within one bf16 ulp of RNE(oracle)
-    want_bits = obf.f64_to_bf16_bits(ref).astype(np.int32)
-    got_bits = y16.view(torch.int16).cpu().numpy().view(np.uint16).astype(np.int32)
-    assert np.abs(got_bits - want_bits).max() <= 1
+    # bf16 output must be the fp32 result rounded once: elementwise within one bf16 rounding (2^-8 relative)
+    # plus the fp32 accumulation error, which scales with the row's largest output, not with the element
+    slack = 2.0 ** -8 * np.abs(ref) + 1e-5 * np.abs(ref).max(axis=1, keepdims=True)
+    assert np.all(np.abs(g16 - ref) <= slack)
+    assert np.all(np.abs(g32 - ref) <= 1e-5 * np.abs(ref).max(axis=1, keepdims=True))
     if end_to_end:
         perm, signs = orp.make_rpbh(d, block, seed)
         qa = oq.quantize_rows(xb, block, perm, signs, oa.boundaries)
