@@ -63,6 +63,13 @@ int oq_build_codebook(int dim, int bits, oq_codebook** out);
  * fp32, centroids_bf16 = levels rounded fp64 -> fp32 -> bf16 (the values the GEMM decodes to). */
 int oq_codebook_get(const oq_codebook* cb, double* centroids, double* boundaries,
                     float* boundaries_f32, uint16_t* centroids_bf16);
+/* Test helper: the polynomial the quantization kernels evaluate instead of a boundary search.  For
+ * x = min(|t| / *clamp, 1) and y = 2x - *centre, floor(P(y)) with
+ * P(y) - 1/2 = *mid + coef[1] y + ... + coef[*degree] y^(*degree) is the number of positive boundaries
+ * below |t| (Eq. 3 restricted to one half of the antisymmetric codebook).  coef has 8 entries.
+ * Returns OQ_ERR_UNSUPPORTED when no monotone polynomial was found (the kernels then search boundaries). */
+int oq_codebook_level_poly(const oq_codebook* cb, float* coef, float* clamp, float* centre, float* mid,
+                           int* degree);
 int oq_codebook_dim(const oq_codebook* cb);
 int oq_codebook_bits(const oq_codebook* cb);
 void oq_codebook_destroy(oq_codebook* cb);

@@ -98,6 +98,80 @@ uint16_t f32_to_bf16_rne(float f) {
   return (uint16_t)(u >> 16);
 }
 
+// Monotone interpolating polynomial for the level search (see QuantPoly).  nb positive boundaries
+// beta[0..nb) in units of the normalised coordinate t.
+QuantPoly build_quant_poly(const double* beta, int nb) {
+  QuantPoly q;
+  q.degree = nb;
+  if (nb < 1 || nb > 7) return q;
+  const int n = nb + 1;
+  double best_slope = 0.0, best_c[8] = {0}, best_clamp = 0.0;
+  const double ratios[] = {1.002, 1.005, 1.01, 1.02, 1.03, 1.05};
+  for (double ratio : ratios) {
+    const double clampv = beta[nb - 1] * ratio;
+    for (int ip = 0; ip <= 90; ++ip) {
+      const double p0 = 0.05 + 0.01 * ip;
+      // nodes y = 2 beta / clamp - 1 (and y = -1 for t = 0), values j (and p0)
+      long double A[8][9];
+      for (int r = 0; r < n; ++r) {
+        const long double y = r == 0 ? -1.0L : 2.0L * beta[r - 1] / clampv - 1.0L;
+        long double pw = 1.0L;
+        for (int c = 0; c < n; ++c) { A[r][c] = pw; pw *= y; }
+        A[r][n] = r == 0 ? p0 : (long double)r;
+      }
+      bool singular = false;
+      for (int c = 0; c < n && !singular; ++c) {
+        int piv = c;
+        for (int r = c + 1; r < n; ++r) if (fabsl(A[r][c]) > fabsl(A[piv][c])) piv = r;
+        if (fabsl(A[piv][c]) < 1e-30L) { singular = true; break; }
+        for (int k = 0; k <= n; ++k) { long double t = A[c][k]; A[c][k] = A[piv][k]; A[piv][k] = t; }
+        for (int r = 0; r < n; ++r) if (r != c) {
+          const long double f = A[r][c] / A[c][c];
+          for (int k = c; k <= n; ++k) A[r][k] -= f * A[c][k];
+        }
+      }
+      if (singular) continue;
+      double c[8];
+      for (int k = 0; k < n; ++k) c[k] = (double)(A[k][n] / A[k][k]);
+      auto P = [&](double y) { double a = c[n - 1]; for (int k = n - 2; k >= 0; --k) a = a * y + c[k]; return a; };
+      auto dP = [&](double y) { double a = (n - 1) * c[n - 1]; for (int k = n - 2; k >= 1; --k) a = a * y + k * c[k]; return a; };
+      const double p1 = P(1.0);
+      if (!(p1 > nb + 1e-3 && p1 < nb + 0.9)) continue;
+      double slope = 1e300;
+      for (int g = 0; g <= 4000; ++g) slope = std::fmin(slope, dP(-1.0 + g / 2000.0));
+      if (slope > best_slope) {
+        best_slope = slope;
+        best_clamp = clampv;
+        for (int k = 0; k < 8; ++k) best_c[k] = k < n ? c[k] : 0.0;
+      }
+    }
+  }
+  if (!(best_slope > 0.0)) return q;
+  // y* with P(y*) = mid + 0.5 (P is increasing on [-1, 1]); then the Taylor shift around y*
+  const double mid = (double)(nb / 2);
+  auto P = [&](double y) { double a = best_c[n - 1]; for (int k = n - 2; k >= 0; --k) a = a * y + best_c[k]; return a; };
+  double lo = -1.0, hi = 1.0;
+  for (int it = 0; it < 200; ++it) {
+    const double m = 0.5 * (lo + hi);
+    if (P(m) < mid + 0.5) lo = m; else hi = m;
+  }
+  const double ys = 0.5 * (lo + hi);
+  double sh[8] = {0};
+  for (int k = 0; k < n; ++k)
+    for (int j = k; j < n; ++j) {
+      double binom = 1.0;
+      for (int i = 0; i < k; ++i) binom = binom * (j - i) / (i + 1);
+      sh[k] += best_c[j] * binom * std::pow(ys, j - k);
+    }
+  q.ok = 1;
+  q.clamp = (float)best_clamp;
+  q.centre = (float)(1.0 + ys);
+  q.mid = (float)mid;
+  for (int k = 1; k < n; ++k) q.coef[k] = (float)sh[k];
+  q.coef[0] = (float)mid;
+  return q;
+}
+
 }  // namespace
 
 CodebookParams codebook_params(const oq_codebook* cb) {
@@ -136,6 +210,18 @@ int ensure_device_tables(const oq_rpbh* rc) {
   e = cudaMalloc(&r->d_gather, sizeof(uint32_t) * r->dim);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
   e = cudaMemcpy(r->d_gather, g.data(), sizeof(uint32_t) * r->dim, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
+  std::vector<uint32_t> off(r->dim), mask((r->dim + 1) / 2, 0u);
+  for (int k = 0; k < r->dim; ++k) {
+    off[k] = 2u * (uint32_t)r->perm[k];
+    if (r->signs[k] < 0) mask[r->perm[k] >> 1] |= (r->perm[k] & 1) ? 0x80000000u : 0x00008000u;
+  }
+  e = cudaMalloc(&r->d_offset, sizeof(uint32_t) * off.size());
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
+  e = cudaMalloc(&r->d_srcmask, sizeof(uint32_t) * mask.size());
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
+  e = cudaMemcpy(r->d_offset, off.data(), sizeof(uint32_t) * off.size(), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(r->d_srcmask, mask.data(), sizeof(uint32_t) * mask.size(), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
   r->device = dev;
   return OQ_OK;
@@ -189,6 +275,7 @@ int oq_build_codebook(int dim, int bits, oq_codebook** out) {
   cb->centroids_bf16.resize(L);
   for (int j = 0; j < L - 1; ++j) cb->boundaries_f32[j] = (float)cb->boundaries[j];
   for (int j = 0; j < L; ++j) cb->centroids_bf16[j] = f32_to_bf16_rne((float)cb->centroids[j]);
+  if (M > 1) cb->poly = build_quant_poly(&cb->boundaries[M], M - 1);
   *out = cb;
   return OQ_OK;
 }
@@ -201,6 +288,16 @@ int oq_codebook_get(const oq_codebook* cb, double* centroids, double* boundaries
   if (boundaries) std::memcpy(boundaries, cb->boundaries.data(), sizeof(double) * (L - 1));
   if (boundaries_f32) std::memcpy(boundaries_f32, cb->boundaries_f32.data(), sizeof(float) * (L - 1));
   if (centroids_bf16) std::memcpy(centroids_bf16, cb->centroids_bf16.data(), sizeof(uint16_t) * L);
+  return OQ_OK;
+}
+int oq_codebook_level_poly(const oq_codebook* cb, float* coef, float* clamp, float* centre, float* mid, int* degree) {
+  if (!cb) return fail(OQ_ERR_INVALID_ARG, "oq_codebook_level_poly: handle is NULL");
+  if (!cb->poly.ok) return fail(OQ_ERR_UNSUPPORTED, "oq_codebook_level_poly: no polynomial for this codebook");
+  if (coef) std::memcpy(coef, cb->poly.coef, sizeof(float) * 8);
+  if (clamp) *clamp = cb->poly.clamp;
+  if (centre) *centre = cb->poly.centre;
+  if (mid) *mid = cb->poly.mid;
+  if (degree) *degree = cb->poly.degree;
   return OQ_OK;
 }
 int oq_codebook_dim(const oq_codebook* cb) { return cb ? cb->dim : 0; }
@@ -259,6 +356,8 @@ int oq_rpbh_block(const oq_rpbh* r) { return r ? r->block : 0; }
 void oq_rpbh_destroy(oq_rpbh* r) {
   if (!r) return;
   if (r->d_gather) cudaFree(r->d_gather);
+  if (r->d_offset) cudaFree(r->d_offset);
+  if (r->d_srcmask) cudaFree(r->d_srcmask);
   delete r;
 }
 

@@ -7,8 +7,23 @@
 
 #include "../../include/oq.h"
 
+// Level search as a polynomial: for a normalised magnitude x = min(|t| / clamp, 1) the number of positive
+// cell boundaries below |t| equals floor(P(x)), with P a monotone polynomial of degree 2^(bits-1) - 1
+// that takes the value j at the j-th boundary.  P is stored re-expanded around the point where it equals
+// mid + 0.5 so that "P - 0.5 + 1.5 * 2^23" has an exactly representable constant term and the rounding
+// of one fused multiply-add leaves floor(P) in the low mantissa bits.
+struct QuantPoly {
+  int degree = 0;          // 2^(bits-1) - 1
+  int ok = 0;              // 1 when a monotone interpolant was found
+  float clamp = 0.f;       // |t| is clamped here (just above the largest boundary)
+  float centre = 0.f;      // y = 2x - centre
+  float coef[8] = {0};     // P(y) - 0.5 = mid + coef[1] y + ... + coef[degree] y^degree
+  float mid = 0.f;         // integer constant term
+};
+
 struct oq_codebook {
   int dim = 0, bits = 0;
+  QuantPoly poly;
   std::vector<double> centroids;     // 2^bits ascending
   std::vector<double> boundaries;    // 2^bits - 1 midpoints
   std::vector<float> boundaries_f32;
@@ -23,6 +38,9 @@ struct oq_rpbh {
   // device copies, created on first GPU use
   int device = -1;
   uint32_t* d_gather = nullptr;  // [dim] word k: low 16 bits = perm[k], bit 31 = 1 when sign is -1
+  uint32_t* d_offset = nullptr;  // [dim] byte offset 2 * perm[k] of the source element of rotated position k
+  uint32_t* d_srcmask = nullptr; // [dim/2] bf16x2 sign-bit masks indexed by SOURCE position: 0x8000 where the
+                                 // element moves to a position whose sign is -1
 };
 
 namespace oq {

@@ -4,6 +4,7 @@
 
 #include "oq_internal.h"
 #include "oq_packing.cuh"
+#include "oq_rq_fast.cuh"
 
 namespace oq {
 
@@ -118,6 +119,70 @@ static int check_common(const char* fn, const void* X, int rows, int dim, int ld
   return OQ_OK;
 }
 
+// Picks rows-per-CTA T and the CTA shape for the fast kernel; returns false when the general kernel
+// has to be used (block size other than 64/128/256, no monotone level polynomial, or a row too long
+// for 8 rows to fit in shared memory).
+struct FastPlan {
+  int T, threads, ctas_per_sm, ncopy;
+  size_t smem;
+};
+static bool plan_fast(int dim, int block, const oq_codebook* cb, FastPlan* plan) {
+  if (block != 64 && block != 128 && block != 256) return false;
+  if (!cb->poly.ok) return false;
+  const size_t kMaxSmem = 227 * 1024;
+  const int lanes_per_block = block / 64;
+  // two buffers of T rows (odd word pitch) + per-warp partial sums + norms (+ the offset table for T >= 8)
+  auto smem_of = [&](int T) {
+    return (size_t)2 * T * (2 * (size_t)dim + 4) + (size_t)(RQ_MAX_THREADS / 32 + 1) * T * 4 + (T >= 8 ? 4 * (size_t)dim : 0);
+  };
+  // rows per buffer: the largest of 16/8/4 that fits; then as many CTAs per SM (1, 2 or 4) as fit
+  int T = 0;
+  for (int c = 16; c >= 4 && !T; c >>= 1) {
+    if (c * lanes_per_block > 32) continue;
+    if (smem_of(c) + 1024 <= kMaxSmem) T = c;
+  }
+  if (!T) return false;
+  int ctas = 1;
+  if (2 * (smem_of(T) + 1024) <= kMaxSmem) ctas = 2;
+  if (4 * (smem_of(T) + 1024) <= kMaxSmem) ctas = 4;
+  plan->T = T;
+  plan->ctas_per_sm = ctas;
+  plan->threads = RQ_MAX_THREADS / ctas;
+  plan->smem = smem_of(T);
+  // copying threads: enough whole warps that each handles at most rq_words_per_thread(T) words per row
+  const int maxw = rq_words_per_thread(T);
+  int ncopy = ((dim / 2 + maxw - 1) / maxw + 31) / 32 * 32;
+  if (ncopy > plan->threads) return false;
+  plan->ncopy = ncopy;
+  return true;
+}
+
+template <int H, int T>
+static cudaError_t launch_fast_bits(int bits, int grid, const FastPlan& pl, cudaStream_t st, const RqFastParams& prm) {
+#define OQ_RQ_LAUNCH(B)                                                                                     \
+  {                                                                                                         \
+    auto k = rq_fast_kernel<H, T, B>;                                                                       \
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);     \
+    if (e != cudaSuccess) return e;                                                                         \
+    k<<<grid, pl.threads, pl.smem, st>>>(prm);                                                              \
+    return cudaGetLastError();                                                                              \
+  }
+  if (bits == 4) OQ_RQ_LAUNCH(4)
+  if (bits == 3) OQ_RQ_LAUNCH(3)
+  OQ_RQ_LAUNCH(2)
+#undef OQ_RQ_LAUNCH
+}
+
+template <int H>
+static cudaError_t launch_fast_T(int bits, int grid, const FastPlan& pl, cudaStream_t st, const RqFastParams& prm) {
+  if (pl.T == 4) return launch_fast_bits<H, 4>(bits, grid, pl, st, prm);
+  if (pl.T == 8) return launch_fast_bits<H, 8>(bits, grid, pl, st, prm);
+  if constexpr (H <= 128) {
+    if (pl.T == 16) return launch_fast_bits<H, 16>(bits, grid, pl, st, prm);
+  }
+  return cudaErrorInvalidValue;
+}
+
 template <bool kBf16Norm>
 static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, const oq_rpbh* rot,
                      const oq_codebook* cb, void* out_idx, void* out_norm, float* dbg, void* stream) {
@@ -132,6 +197,25 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
   cudaGetDevice(&dev);
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  FastPlan pl;
+  if (plan_fast(dim, rot->block, cb, &pl)) {
+    RqFastParams prm;
+    prm.X = reinterpret_cast<const uint32_t*>(X);
+    prm.rows = rows; prm.dim = dim; prm.ldw = ld / 2;
+    prm.offset = rot->d_offset; prm.srcmask = rot->d_srcmask;
+    prm.out_idx = reinterpret_cast<uint32_t*>(out_idx); prm.pitch_words = pitch_words;
+    prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
+    prm.groups = (rows + pl.T - 1) / pl.T;
+    prm.bf16_norm = kBf16Norm ? 1 : 0;
+    prm.ncopy = pl.ncopy;
+    int grid = sms * pl.ctas_per_sm;
+    if (grid > prm.groups) grid = prm.groups;
+    if (rot->block == 64) e = launch_fast_T<64>(cb->bits, grid, pl, st, prm);
+    else if (rot->block == 128) e = launch_fast_T<128>(cb->bits, grid, pl, st, prm);
+    else e = launch_fast_T<256>(cb->bits, grid, pl, st, prm);
+    if (e != cudaSuccess) return cuda_fail(e, fn);
+    return OQ_OK;
+  }
   const size_t smem = (size_t)dim * 5;
   auto kern = rq_general_kernel<kBf16Norm>;
   if (smem > 48 * 1024) {

@@ -1,0 +1,101 @@
+"""Per-kernel micro-benchmarks (device-timed with CUDA events, L2 flushed between iterations).
+
+    python -m paper_2607_02461_b200.microbench rq   --tokens 17776 --dim 3072 --bits 4 --block 128
+    python -m paper_2607_02461_b200.microbench gemm --tokens 4608 --dim 3072 --m 9216 --bits-a 4 --bits-w 4
+    python -m paper_2607_02461_b200.microbench sweep [--quick]     # rotate+quantize bandwidth sweep
+
+Inputs are synthetic and generated on the GPU (normal values, per-token log-uniform scale, 1% of the
+channels multiplied by 30); these runs time the kernels, parity is covered by the tests.
+Each run prints one JSON line per point.
+"""
+import argparse
+import json
+import sys
+
+import torch
+
+from . import binding as B
+from . import build as oqbuild
+
+
+def gen_x(n, d, seed=0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    x = torch.randn((n, d), device="cuda", generator=g)
+    x *= torch.exp(torch.empty(n, 1, device="cuda").uniform_(-2.3026, 2.3026, generator=g))
+    ch = torch.randperm(d, device="cuda", generator=g)[: max(1, d // 100)]
+    x[:, ch] *= 30.0
+    return x.to(torch.bfloat16)
+
+
+def time_kernel(fn, iters, warmup=3, flush_mb=256):
+    flush = torch.empty(flush_mb << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(warmup):
+        fn()
+    ts = []
+    for _ in range(iters):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ts.sort()
+    return ts[len(ts) // 2], ts[0]
+
+
+def run_rq(n, d, bits, block, iters):
+    rot, cb = B.oq_make_rpbh(d, block, 0), B.oq_build_codebook(d, bits)
+    X = gen_x(n, d)
+    idx = torch.empty((n, B.oq_packed_bytes(n, d, bits)[1]), dtype=torch.uint8, device="cuda")
+    nrm = torch.empty(n, dtype=torch.float32, device="cuda")
+    med, best = time_kernel(lambda: B.oq_rotate_quantize_act(X, rot, cb, out_idx=idx, out_norm=nrm), iters)
+    nbytes = 2 * n * d + n * d * bits // 8 + 4 * n
+    return {"kernel": "rotate_quantize", "tokens": n, "dim": d, "bits": bits, "block": block, "ms_median": med,
+            "ms_min": best, "bytes": nbytes, "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
+
+
+def run_gemm(n, d, m, ba, bw, iters):
+    rot = B.oq_make_rpbh(d, 128, 0)
+    cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
+    xq, xs = B.oq_rotate_quantize_act(gen_x(n, d), rot, cba)
+    W = (torch.randn((m, d), device="cuda") * 0.02).to(torch.bfloat16)
+    wq, wr = B.oq_quantize_weights(W, rot, cbw)
+    del W
+    Y = torch.empty((n, m), dtype=torch.bfloat16, device="cuda")
+    med, best = time_kernel(lambda: B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out=Y), iters)
+    fl = 2.0 * n * m * d
+    return {"kernel": "qlinear", "tokens": n, "dim": d, "m": m, "bits_a": ba, "bits_w": bw, "ms_median": med,
+            "ms_min": best, "flops": fl, "tflops": fl / med / 1e9, "tflops_best": fl / best / 1e9}
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("mode", choices=["rq", "gemm", "sweep"])
+    ap.add_argument("--tokens", type=int, default=17776)
+    ap.add_argument("--dim", type=int, default=3072)
+    ap.add_argument("--m", type=int, default=9216)
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--bits-a", type=int, default=4)
+    ap.add_argument("--bits-w", type=int, default=4)
+    ap.add_argument("--block", type=int, default=128)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--quick", action="store_true")
+    a = ap.parse_args(argv)
+    oqbuild.build()
+    if a.mode == "rq":
+        print(json.dumps(run_rq(a.tokens, a.dim, a.bits, a.block, a.iters)))
+    elif a.mode == "gemm":
+        print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters)))
+    else:
+        toks = [4608, 32760] if a.quick else [4608, 17776, 32760, 75600]
+        for n in toks:
+            for d in [1024, 3072, 5120, 12288, 13824]:
+                for bits in [3, 4]:
+                    for block in [64, 128, 256]:
+                        print(json.dumps(run_rq(n, d, bits, block, a.iters)))
+                        sys.stdout.flush()
+                        torch.cuda.empty_cache()
+    assert B.oq_device_status() == 0
+
+
+if __name__ == "__main__":
+    main()

@@ -54,17 +54,20 @@ def check_rows(xb, block, seed, bits, weights=False, rows=None):
     gi, ri = idx[sel].astype(np.int32), ref["idx"].astype(np.int32)
     flips = np.argwhere(gi != ri)
     tmax = np.abs(ref["unit"]).max(axis=1)
+    ties = 0
     for r, k in flips:
         assert abs(gi[r, k] - ri[r, k]) == 1
         beta = ocbk.boundaries[min(gi[r, k], ri[r, k])]
         assert abs(ref["unit"][r, k] - beta) <= BAND * tmax[r]
-    return len(flips) / gi.size
+        ties += ref["unit"][r, k] == beta          # exactly on a boundary: both neighbours are nearest (Eq. 3)
+    return (len(flips) - ties) / gi.size
 
 
 @pytest.mark.parametrize("bits", [4, 3, 2])
-@pytest.mark.parametrize("d,block", [(1024, 128), (384, 64), (768, 256), (1024, 1024), (128, 8)])
+@pytest.mark.parametrize("d,block", [(1024, 128), (384, 64), (768, 256), (1024, 1024), (128, 8), (3072, 128),
+                                     (5120, 256), (5120, 64), (13824, 128), (12288, 256), (1024, 256)])
 def test_activation_rows_match_oracle(d, block, bits):
-    xb = synth.activations(67, d, seed=1000 + bits)        # 67 rows: ragged against any row tiling
+    xb = synth.activations(67 if d < 8000 else 21, d, seed=1000 + bits)   # ragged against any row tiling
     rate = check_rows(xb, block, 0, bits)
     assert rate <= 1e-4
 
@@ -90,7 +93,7 @@ def test_degenerate_tokens_and_strided_input():
     x[3, ::2] = -2.0 ** -120          # tiny values: squares underflow in fp32
     x[4, :] = np.random.default_rng(0).standard_normal(d) * 1e4
     xb = synth.to_bf16_bits(x)
-    assert check_rows(xb, 128, 3, 4, rows=[0, 1, 2, 4]) <= 2e-3   # exact zeros sit on the middle boundary (ties)
+    assert check_rows(xb, 128, 3, 4, rows=[0, 1, 2, 4]) <= 1e-4   # exact zeros sit on the middle boundary (ties)
     rot, cb = B.oq_make_rpbh(d, 128, 3), B.oq_build_codebook(d, 4)
     # leading dimension larger than dim
     wide = torch.zeros((5, d + 64), dtype=torch.bfloat16, device="cuda")
@@ -99,7 +102,8 @@ def test_degenerate_tokens_and_strided_input():
     b_idx, b_norm = B.oq_rotate_quantize_act(_dev(xb), rot, cb)
     assert torch.equal(a_idx, b_idx) and torch.equal(a_norm, b_norm)
     assert a_norm[0].item() == 0.0
-    assert torch.all(B.oq_unpack_indices(a_idx, 5, d, 4)[0] == 7)
+    z = B.oq_unpack_indices(a_idx, 5, d, 4)[0]
+    assert torch.all((z == 7) | (z == 8))           # t = 0 is equidistant from the two middle levels
 
 
 def test_empty_and_bad_arguments():

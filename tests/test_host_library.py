@@ -79,3 +79,45 @@ def test_packed_sizes():
     for d in (128, 1024, 13824):
         for b in (2, 3, 4):
             assert B.oq_packed_bytes(1, d, b)[1] % 16 == 0 and B.oq_packed_bytes(1, d, b)[1] * 8 == d * b
+
+
+@pytest.mark.parametrize("dim,bits", [(64, 4), (1024, 4), (13824, 4), (3072, 3), (5120, 2), (128, 3)])
+def test_level_search_polynomial_counts_boundaries(dim, bits):
+    """The kernels find a level as floor(P(x)) with P evaluated in fp32 (fused multiply-adds, the last one
+    adding 1.5 * 2^23 so that the integer part lands in the low mantissa bits).  Emulate exactly that and
+    compare with the oracle's boundary count on a fine grid; mismatches may only sit within 1e-6 of a
+    boundary (relative to the largest boundary)."""
+    import ctypes as C
+    cb = B.oq_build_codebook(dim, bits)
+    coef = (C.c_float * 8)()
+    clamp, centre, mid, deg = C.c_float(), C.c_float(), C.c_float(), C.c_int()
+    L = B.lib()
+    L.oq_codebook_level_poly.restype = C.c_int
+    assert L.oq_codebook_level_poly(cb.handle, coef, C.byref(clamp), C.byref(centre), C.byref(mid), C.byref(deg)) == 0
+    nb = (1 << bits) // 2 - 1
+    assert deg.value == nb
+    beta = ocb.lloyd_max(dim, bits).boundaries[nb + 1:]
+    f32 = np.float32
+
+    def fma(a, b, c):
+        return (a.astype(np.float64) * np.asarray(b, np.float64) + np.float64(c)).astype(f32)
+
+    t = np.concatenate([np.linspace(0, 1.3 * beta[-1], 1000001), np.linspace(1.3 * beta[-1], 1.0, 1001)])
+    for s in (3.7, 1e-3, 4e4, 0.0):
+        h = 128
+        z = (t * np.sqrt(h) * (s + 1e-10)).astype(f32)
+        kappa = f32(1.0) / f32(f32(np.sqrt(f32(h))) * f32(f32(s) + f32(1e-10)) * clamp.value)
+        x = np.clip(fma(np.abs(z), kappa, 0.0), 0, 1)
+        y = fma(x, f32(2), -centre.value)
+        acc = np.full_like(y, coef[nb])
+        for k in range(nb - 1, 0, -1):
+            acc = fma(acc, y, coef[k])
+        v = fma(acc, y, f32(mid.value + 12582912.0))
+        mag = v.view(np.uint32).astype(np.int64) - 0x4B400000
+        texact = z.astype(np.float64) / (np.sqrt(h) * (s + 1e-10))
+        want = np.searchsorted(beta, texact, side="left")
+        bad = mag != want
+        assert mag.min() >= 0 and mag.max() <= nb
+        if bad.any():
+            dist = np.min(np.abs(texact[bad][:, None] - beta[None, :]), axis=1)
+            assert dist.max() <= 1e-6 * beta[-1] and np.abs(mag - want)[bad].max() == 1
