@@ -12,17 +12,19 @@ namespace oq {
 
 namespace {
 
-constexpr int BM = 128;   // tokens per tile   (MMA M, TMEM lanes)
-constexpr int BN = 256;   // features per tile (MMA N, TMEM columns)
+constexpr int BM = 256;   // tokens per tile: two MMAs of M = 128, one accumulator each
+constexpr int BN = 256;   // features per tile (MMA N)
 constexpr int BK = 64;    // coordinates per stage: 64 bf16 = one 128-byte swizzled row
-constexpr int STAGES = 2;
-constexpr int THREADS = 256;
+constexpr int STAGES = 3;
+constexpr int DECODE_THREADS = 512;            // 16 warps decode and, after the last stage, run the epilogue
+constexpr int THREADS = DECODE_THREADS + 32;   // + one warp whose lane 0 issues the MMAs
+constexpr int TMEM_COLS = 512;                 // 2 accumulators x 256 fp32 columns
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s: a wait that lasts longer reports and gives up
 
-enum { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC = 3 };
+enum { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_FULL = 3, WAIT_ACC_EMPTY = 4 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -89,11 +91,30 @@ __device__ __forceinline__ Tables make_tables(const CodebookParams& cb) {
 }
 
 // Decodes 32 consecutive coordinates (BITS words of one packed row) into four 16-byte chunks of bf16.
+// Raw packed words of 32 coordinates of one row (BITS words), fetched ahead of their use.
 template <int BITS>
-__device__ __forceinline__ void decode32(const uint32_t* __restrict__ src, const Tables& t, uint4 out[4]) {
+struct Raw {
+  uint32_t w[BITS];
+};
+template <int BITS>
+__device__ __forceinline__ Raw<BITS> load_raw(const uint32_t* __restrict__ src) {
+  Raw<BITS> r;
   if (BITS == 4) {
-    const uint4 w4 = *reinterpret_cast<const uint4*>(src);
-    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+    r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[BITS - 1] = v.w;
+  } else if (BITS == 3) {
+    r.w[0] = __ldg(src); r.w[1] = __ldg(src + 1); r.w[2] = __ldg(src + 2);
+  } else {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(src));
+    r.w[0] = v.x; r.w[1] = v.y;
+  }
+  return r;
+}
+
+template <int BITS>
+__device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, uint4 out[4]) {
+  if (BITS == 4) {
+    const uint32_t* w = raw.w;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const uint32_t sel = w[q] & 0x77777777u;
@@ -104,13 +125,8 @@ __device__ __forceinline__ void decode32(const uint32_t* __restrict__ src, const
                           prmt(loB, hiB, 0x7362u));
     }
   } else {
-    uint32_t mw[2], s;
-    if (BITS == 3) {
-      mw[0] = src[0]; mw[1] = src[1]; s = src[2];
-    } else {
-      const uint2 v = *reinterpret_cast<const uint2*>(src);
-      mw[0] = v.x; mw[1] = v.x; s = v.y;
-    }
+    const uint32_t mw[2] = {raw.w[0], raw.w[BITS == 3 ? 1 : 0]};
+    const uint32_t s = raw.w[BITS - 1];
     uint32_t r[16];
 #pragma unroll
     for (int G = 0; G < 8; ++G) {
@@ -143,36 +159,36 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = 256.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
 template <int BITS_A, int BITS_W, bool F32_OUT>
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(THREADS, 1)
 qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm, int n_tokens,
                const uint32_t* __restrict__ Wq, const __nv_bfloat16* __restrict__ w_norm, int m, int dim,
                CodebookParams cba, CodebookParams cbw, void* __restrict__ Y, int ldy, int* status) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int i0 = blockIdx.x * BN;   // first feature of the tile
-  const int n0 = blockIdx.y * BM;   // first token of the tile
-  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES), accbar = smem_u32(bars + 2 * STAGES);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
+  const uint32_t accfull = smem_u32(bars + 2 * STAGES), accempty = smem_u32(bars + 2 * STAGES + 1);
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full0 + 8 * s, THREADS);
-      mbar_init(empty0 + 8 * s, 1);
+      mbar_init(full0 + 8 * s, DECODE_THREADS);   // every decoding thread arrives once per stage
+      mbar_init(empty0 + 8 * s, 1);               // tcgen05.commit arrives once the MMAs have read the stage
     }
-    mbar_init(accbar, 1);
+    mbar_init(accfull, 1);                        // tcgen05.commit after the last stage of a tile
+    mbar_init(accempty, DECODE_THREADS);          // every epilogue thread arrives after reading its columns
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -180,109 +196,149 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
 
-  const Tables ta = make_tables(cba), tw = make_tables(cbw);
-  const int pitch_a = dim / 32 * BITS_A, pitch_w = dim / 32 * BITS_W;   // words per packed row
-  // this thread's decode tasks: one (row, half) of A and two of B per stage
-  const int a_row = tid >> 1, a_half = tid & 1;
-  const int a_src_row = min(n0 + a_row, n_tokens - 1);
-  const uint32_t* a_src = Aq + (size_t)a_src_row * pitch_a + a_half * BITS_A;
-  const uint32_t* b_src[2];
-  int b_row[2];
-#pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    b_row[j] = (tid >> 1) + j * 128;
-    b_src[j] = Wq + (size_t)min(i0 + b_row[j], m - 1) * pitch_w + a_half * BITS_W;
-  }
-
   const int kblocks = dim / BK;
-  for (int kb = 0; kb < kblocks; ++kb) {
-    const int st = kb % STAGES;
-    const uint32_t use = kb / STAGES;
-    if (kb >= STAGES) mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, WAIT_EMPTY);
-    unsigned char* As = smem + st * STAGE_BYTES;
-    unsigned char* Bs = As + A_BYTES;
-    uint4 v[4];
-    decode32<BITS_A>(a_src + (size_t)kb * 2 * BITS_A, ta, v);
-    store_half(As, a_row, a_half, v);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      decode32<BITS_W>(b_src[j] + (size_t)kb * 2 * BITS_W, tw, v);
-      store_half(Bs, b_row[j], a_half, v);
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
-    mbar_arrive(full0 + 8 * st);
-    if (tid == 0) {
-      mbar_wait(full0 + 8 * st, use & 1, abort_flag, status, WAIT_FULL);
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint64_t da = smem_desc(smem_u32(As)), db = smem_desc(smem_u32(Bs));
-#pragma unroll
-      for (int k4 = 0; k4 < BK / 16; ++k4) {
-        const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
-        asm volatile(
-            "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-            " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-            ::"r"(tmem), "l"(da + 2 * k4), "l"(db + 2 * k4), "r"(IDESC), "r"(acc)
-            : "memory");
-      }
-      // arrives on empty[st] once every MMA issued so far has finished reading shared memory
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(empty0 + 8 * st) : "memory");
-    }
-  }
-  if (tid == 0)
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(accbar) : "memory");
-  mbar_wait(accbar, 0, abort_flag, status, WAIT_ACC);
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  __syncwarp();   // the per-thread wait loops above may leave the warp diverged; tcgen05.ld is warp-collective
+  const int tiles_n = (n_tokens + BM - 1) / BM, tiles_m = (m + BN - 1) / BN;
+  const int ntiles = tiles_n * tiles_m;   // token tiles vary fastest: CTAs running together share weight rows
 
-  // Epilogue: warp w reads TMEM lanes 32*(w%4).., columns 128*(w/4)..; lane = one token row.
-  {
-    const int row = n0 + (warp & 3) * 32 + lane;
-    const float s = row < n_tokens ? a_norm[row] : 0.f;
+  if (warp == DECODE_THREADS / 32) {
+    // ------------------------------- MMA issuer (one thread) -------------------------------
+    if (lane == 0) {
+      uint32_t g = 0, lt = 0;
+      for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+        if (lt > 0) mbar_wait(accempty, (lt - 1) & 1, abort_flag, status, WAIT_ACC_EMPTY);   // epilogue drained TMEM
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int kb = 0; kb < kblocks; ++kb, ++g) {
+          const uint32_t st = g % STAGES, use = g / STAGES;
+          mbar_wait(full0 + 8 * st, use & 1, abort_flag, status, WAIT_FULL);
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = smem_u32(smem + st * STAGE_BYTES);
+          const uint64_t da0 = smem_desc(a_addr), da1 = smem_desc(a_addr + 128 * 128), db = smem_desc(a_addr + A_BYTES);
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 16; ++k4) {
+            const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
+            asm volatile(
+                "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                ::"r"(tmem), "l"(da0 + 2 * k4), "l"(db + 2 * k4), "r"(IDESC), "r"(acc) : "memory");
+            asm volatile(
+                "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                ::"r"(tmem + BN), "l"(da1 + 2 * k4), "l"(db + 2 * k4), "r"(IDESC), "r"(acc) : "memory");
+          }
+          // arrives on empty[st] once every MMA issued so far has finished reading shared memory
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(empty0 + 8 * st) : "memory");
+        }
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(accfull) : "memory");
+      }
+    }
+  } else {
+    // ------------------- decoders (all 16 warps), then the epilogue of the tile -------------------
+    const Tables ta = make_tables(cba), tw = make_tables(cbw);
+    const int pitch_a = dim / 32 * BITS_A, pitch_w = dim / 32 * BITS_W;   // words per packed row
+    const int row = tid >> 1, half = tid & 1;          // one (row, 32-coordinate half) of A and one of B per stage
+    uint32_t g = 0, lt = 0;
+    const uint32_t* a_src = nullptr;
+    const uint32_t* b_src = nullptr;
+    auto set_tile = [&](int tile) {
+      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
+      a_src = Aq + (size_t)min(n0 + row, n_tokens - 1) * pitch_a + half * BITS_A;   // rows past the end re-read the last
+      b_src = Wq + (size_t)min(i0 + row, m - 1) * pitch_w + half * BITS_W;          // row; their outputs are never stored
+    };
+    Raw<BITS_A> ra;
+    Raw<BITS_W> rb;
+    if ((int)blockIdx.x < ntiles) {
+      set_tile(blockIdx.x);
+      ra = load_raw<BITS_A>(a_src);
+      rb = load_raw<BITS_W>(b_src);
+    }
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
+      for (int kb = 0; kb < kblocks; ++kb, ++g) {
+        const uint32_t st = g % STAGES, use = g / STAGES;
+        // fetch the next stage's packed words before decoding this one
+        Raw<BITS_A> na = ra;
+        Raw<BITS_W> nb = rb;
+        if (kb + 1 < kblocks) {
+          na = load_raw<BITS_A>(a_src + (size_t)(kb + 1) * 2 * BITS_A);
+          nb = load_raw<BITS_W>(b_src + (size_t)(kb + 1) * 2 * BITS_W);
+        } else if (tile + (int)gridDim.x < ntiles) {
+          set_tile(tile + gridDim.x);
+          na = load_raw<BITS_A>(a_src);
+          nb = load_raw<BITS_W>(b_src);
+        }
+        if (use > 0) mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, WAIT_EMPTY);
+        unsigned char* As = smem + st * STAGE_BYTES;
+        uint4 v[4];
+        decode32<BITS_A>(ra, ta, v);
+        store_half(As, row, half, v);
+        decode32<BITS_W>(rb, tw, v);
+        store_half(As + A_BYTES, row, half, v);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+        mbar_arrive(full0 + 8 * st);
+        ra = na;
+        rb = nb;
+      }
+      // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .., columns 128 (w / 4) ..; lane = one token row ----
+      mbar_wait(accfull, lt & 1, abort_flag, status, WAIT_ACC_FULL);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      __syncwarp();   // the per-thread wait loops may leave the warp diverged; tcgen05.ld is warp-collective
+      {
+        const int cg = warp >> 2;                        // 128-column group: accumulator cg / 2, feature half cg % 2
+        const int trow = n0 + (cg >> 1) * 128 + (warp & 3) * 32 + lane;
+        const float s = trow < n_tokens ? a_norm[trow] : 0.f;
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
-      const int col0 = (warp >> 2) * 128 + c * 32;
-      uint32_t r[32];
-      const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
-      asm volatile(
-          "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-          "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-            "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-            "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-            "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-          : "r"(taddr)
-          : "memory");
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (row < n_tokens) {
+        for (int c = 0; c < 4; ++c) {
+          const int fcol = (cg & 1) * 128 + c * 32;      // feature offset inside the tile
+          uint32_t r[32];
+          const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(cg * 128 + c * 32);
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+              "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+                "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+              : "r"(taddr)
+              : "memory");
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (trow < n_tokens) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {   // 8 features per group
-          const int i = i0 + col0 + g * 8;
-          if (i < m) {
-            float y[8];
+            for (int g8 = 0; g8 < 4; ++g8) {   // 8 features per group
+              const int i = i0 + fcol + g8 * 8;
+              if (i < m) {
+                const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));   // 8 bf16 row norms
+                const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
+                float y[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-              y[j] = (__uint_as_float(r[g * 8 + j]) * s) * __bfloat162float(w_norm[i + j]);
-            if (F32_OUT) {
-              float* dst = reinterpret_cast<float*>(Y) + (size_t)row * ldy + i;
-              *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
-              *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
-            } else {
-              __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
-              __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
-              uint4 pk;
-              pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-              pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-              *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(Y) + (size_t)row * ldy + i) = pk;
+                for (int j = 0; j < 4; ++j) {
+                  y[2 * j] = (__uint_as_float(r[g8 * 8 + 2 * j]) * s) * __uint_as_float(rw[j] << 16);
+                  y[2 * j + 1] = (__uint_as_float(r[g8 * 8 + 2 * j + 1]) * s) * __uint_as_float(rw[j] & 0xFFFF0000u);
+                }
+                if (F32_OUT) {
+                  float* dst = reinterpret_cast<float*>(Y) + (size_t)trow * ldy + i;
+                  *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
+                  *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
+                } else {
+                  __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
+                  __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
+                  uint4 pk;
+                  pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                  pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                  *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(Y) + (size_t)trow * ldy + i) = pk;
+                }
+              }
             }
           }
         }
       }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(accempty);   // this thread's TMEM reads are done: the next tile may overwrite the accumulators
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
 template <int BA, int BW>
@@ -325,12 +381,17 @@ extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens
   if (n_tokens == 0 || m == 0) return OQ_OK;
   if (!Xq_idx || !Xq_norm || !Wq_idx || !Wq_norm_bf16 || !Y) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: NULL buffer");
   if (ldy < m) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: ldy smaller than m");
-  if (ldy % 8 || !aligned16(Xq_idx) || !aligned16(Wq_idx) || !aligned16(Y))
+  if (ldy % 8 || !aligned16(Xq_idx) || !aligned16(Wq_idx) || !aligned16(Y) || !aligned16(Wq_norm_bf16))
     return fail(OQ_ERR_ALIGNMENT, "oq_qlinear: pointers must be 16-byte aligned and ldy a multiple of 8");
   int* status = device_status_word();
   if (!status) return fail(OQ_ERR_CUDA, "oq_qlinear: cannot allocate the device status word");
   const CodebookParams ca = codebook_params(cb_a), cw = codebook_params(cb_w);
-  dim3 grid((m + BN - 1) / BN, (n_tokens + BM - 1) / BM);
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaError_t ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (ce != cudaSuccess) return cuda_fail(ce, "cudaDeviceGetAttribute");
+  const int ntiles = ((m + BN - 1) / BN) * ((n_tokens + BM - 1) / BM);
+  dim3 grid(ntiles < sms ? ntiles : sms);   // persistent: one CTA per SM walks the tiles
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const uint32_t* A = reinterpret_cast<const uint32_t*>(Xq_idx);
   const uint32_t* W = reinterpret_cast<const uint32_t*>(Wq_idx);
