@@ -145,6 +145,30 @@ int oq_linear_forward_host(const void* X_host_bf16, int n_tokens, int dim, const
                            const oq_codebook* cb_w, void* Y_host_bf16, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* Whole online layer on DEVICE buffers without any allocation.  The paper has no counterpart: this is a
+ * variant of the layer call for callers that cannot obtain device memory when they need the layer
+ * evaluated -- a serving loop confined to a memory budget fixed at start-up, a thread that must not block on
+ * the allocator, a process whose memory pool is already frozen.  It runs oq_rotate_quantize_act and then
+ * oq_qlinear; the packed activations, their norms and the status word that bounded device-side waits
+ * report to are kept in a scratch array that is compiled into the library (about 8.1 MiB of device memory
+ * on every GPU that loads the library, held until the process exits).  The call performs no cudaMalloc /
+ * cudaFree and calls no allocating library routine.
+ *   X_bf16 dev [n_tokens][ldx] bf16;  Wq_idx / Wq_norm_bf16 dev, from oq_quantize_weights;
+ *   Y dev [n_tokens][ldy] of y_dtype, written.  Arguments as for the two calls it wraps.
+ * Limits: n_tokens <= 32768 and oq_packed_bytes(n_tokens, dim, bits_a) <= 8 MiB, otherwise OQ_ERR_NOMEM
+ * with a message that states both sizes.  `rot` must already have been used by an ordinary GPU call
+ * (oq_quantize_weights does that), because creating its device tables allocates; otherwise
+ * OQ_ERR_INVALID_ARG.
+ * The first call on a device looks up the scratch array's device address and clears its status word with a
+ * blocking memset: make that first call before starting any stream capture.
+ * All calls on a device share the one scratch array, which keeps the previous call's contents: two calls
+ * whose kernels may overlap on the GPU (different streams) race on it -- serialise them.  Nothing in the
+ * scratch needs clearing between calls (every byte that is read was written by the same call); the status
+ * word is sticky until oq_device_status reads it. */
+int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                              const oq_codebook* cb_a, const void* Wq_idx, const void* Wq_norm_bf16, int m,
+                              const oq_codebook* cb_w, void* Y, int ldy, int y_dtype, void* stream);
+
 /* Test helper: expand packed indices to one byte per coordinate, out dev [rows][dim] uint8, logical level
  * numbers in rotated-coordinate order. */
 int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream);

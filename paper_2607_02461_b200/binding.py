@@ -44,6 +44,7 @@ def lib():
             "oq_quantize_weights": (i, [vp, i, i, i, vp, vp, vp, vp, vp, vp]),
             "oq_qlinear": (i, [vp, vp, i, vp, vp, vp, i, vp, i, vp, i, i, vp]),
             "oq_unpack_indices": (i, [vp, i, i, i, vp, vp]),
+            "oq_linear_forward_noalloc": (i, [vp, i, i, i, vp, vp, vp, vp, i, vp, vp, i, i, vp]),
             "oq_forward_workspace_bytes": (i, [i, i, i, i, C.POINTER(sz)]),
             "oq_linear_forward_host": (i, [vp, i, i, vp, vp, vp, vp, i, vp, vp, vp, sz, vp]),
             "oq_device_status": (i, [C.POINTER(i)]),
@@ -180,6 +181,19 @@ def oq_linear_forward_host(X_host, rot, cb_a, Wq_idx, Wq_norm, cb_w, Y_host, wor
     _check(lib().oq_linear_forward_host(_ptr(X_host), n, d, rot.handle, cb_a.handle, _ptr(Wq_idx), _ptr(Wq_norm), m,
                                         cb_w.handle, _ptr(Y_host), _ptr(workspace), workspace.numel(), _stream()))
     return Y_host
+
+
+def oq_linear_forward_noalloc(X, rot, cb_a, Wq_idx, Wq_norm, cb_w, out):
+    """Allocation-free layer call: X CUDA bf16 [N, d], `out` a preallocated CUDA [N, m] bf16 or fp32 tensor.
+    Nothing is allocated here or in the library (the hand-over buffers are a static device array)."""
+    import torch
+    n, d = X.shape
+    m = Wq_idx.shape[0]
+    ydt = OQ_F32 if out.dtype == torch.float32 else OQ_BF16
+    _check(lib().oq_linear_forward_noalloc(_ptr(X), n, d, X.stride(0) if n > 1 else d, rot.handle, cb_a.handle,
+                                           _ptr(Wq_idx), _ptr(Wq_norm), m, cb_w.handle, _ptr(out),
+                                           out.stride(0) if n > 1 else m, ydt, _stream()))
+    return out
 
 
 def oq_unpack_indices(idx, rows, dim, bits):

@@ -380,6 +380,14 @@ int oq_device_status(int* status) {
   if (!w) return fail(OQ_ERR_CUDA, "oq_device_status: no status word (no usable device?)");
   e = cudaMemcpy(status, w, sizeof(int), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+  if (*status == 0) {
+    // the allocation-free entry point keeps its own status word
+    if (int* w2 = noalloc_status_word()) {
+      e = cudaMemcpy(status, w2, sizeof(int), cudaMemcpyDeviceToHost);
+      if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+      if (*status != 0) cudaMemset(w2, 0, sizeof(int));
+    }
+  }
   if (*status != 0) {
     cudaMemset(w, 0, sizeof(int));
     return fail(OQ_ERR_DEVICE_TIMEOUT, "a bounded device-side wait gave up; status code " + std::to_string(*status));

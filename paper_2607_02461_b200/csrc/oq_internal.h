@@ -60,6 +60,12 @@ CodebookParams codebook_params(const oq_codebook* cb);
 // Device status word (bounded waits report here).
 int* device_status_word();   // device pointer (allocated on first use), or nullptr on failure
 
+int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
+                   const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y,
+                   int ldy, int y_dtype, int* status, void* stream);
+// Status word of the allocation-free entry point on the current device, or nullptr before its first call.
+int* noalloc_status_word();
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace oq

@@ -373,11 +373,13 @@ int launch_bits(bool f32, int bn, dim3 grid, cudaStream_t st, const uint32_t* Aq
 }  // namespace
 }  // namespace oq
 
-using namespace oq;
+namespace oq {
 
-extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
-                          const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim,
-                          void* Y, int ldy, int y_dtype, void* stream) {
+// Validates and launches; `status` is the device word that bounded waits report to (NULL: the library's own
+// word, allocated on first use).
+int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
+                   const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y,
+                   int ldy, int y_dtype, int* status, void* stream) {
   if (!cb_a || !cb_w) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: NULL codebook");
   if (n_tokens < 0 || m < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: bad sizes");
   if (cb_a->dim != dim || cb_w->dim != dim) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: codebook dim differs from dim");
@@ -391,7 +393,7 @@ extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens
   if (ldy < m) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear: ldy smaller than m");
   if (ldy % 8 || !aligned16(Xq_idx) || !aligned16(Wq_idx) || !aligned16(Y) || !aligned16(Wq_norm_bf16))
     return fail(OQ_ERR_ALIGNMENT, "oq_qlinear: pointers must be 16-byte aligned and ldy a multiple of 8");
-  int* status = device_status_word();
+  if (!status) status = device_status_word();
   if (!status) return fail(OQ_ERR_CUDA, "oq_qlinear: cannot allocate the device status word");
   const CodebookParams ca = codebook_params(cb_a), cw = codebook_params(cb_w);
   int dev = 0, sms = 0;
@@ -416,4 +418,13 @@ extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens
   OQ_CASE(4, 4) OQ_CASE(3, 3) OQ_CASE(4, 2) OQ_CASE(3, 2) OQ_CASE(4, 3) OQ_CASE(2, 2) OQ_CASE(3, 4) OQ_CASE(2, 4) OQ_CASE(2, 3)
 #undef OQ_CASE
   return fail(OQ_ERR_UNSUPPORTED, "oq_qlinear: unsupported bit-width pair");
+}
+
+}  // namespace oq
+
+extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
+                          const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim,
+                          void* Y, int ldy, int y_dtype, void* stream) {
+  return oq::qlinear_launch(Xq_idx, Xq_norm, n_tokens, cb_a, Wq_idx, Wq_norm_bf16, m, cb_w, dim, Y, ldy, y_dtype,
+                            nullptr, stream);
 }
