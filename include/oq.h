@@ -178,6 +178,12 @@ int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out
  * OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
 int oq_device_status(int* status);
 
+/* Self-test of the bounded device-side waits the GEMM pipeline is built on: launches one thread that waits
+ * about a millisecond on a barrier nobody arrives at.  The wait gives up by itself (the kernel ends
+ * normally, nothing hangs or traps) and records code 9; the following oq_device_status() must return
+ * OQ_ERR_DEVICE_TIMEOUT with *status == 9 and leave the word clear again. */
+int oq_selftest_bounded_wait(void* stream);
+
 const char* oq_last_error(void);
 const char* oq_version(void);
 

@@ -48,6 +48,7 @@ def lib():
             "oq_forward_workspace_bytes": (i, [i, i, i, i, C.POINTER(sz)]),
             "oq_linear_forward_host": (i, [vp, i, i, vp, vp, vp, vp, i, vp, vp, vp, sz, vp]),
             "oq_device_status": (i, [C.POINTER(i)]),
+            "oq_selftest_bounded_wait": (i, [vp]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
         for name, (res, args) in sig.items():
@@ -209,6 +210,10 @@ def oq_device_status():
     if code not in (0, 5):
         _check(code)
     return s.value
+
+
+def oq_selftest_bounded_wait():
+    _check(lib().oq_selftest_bounded_wait(_stream()))
 
 
 def oq_version():

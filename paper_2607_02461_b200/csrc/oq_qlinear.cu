@@ -24,7 +24,7 @@ constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s: a wait that lasts longer reports and gives up
 
-enum { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_FULL = 3, WAIT_ACC_EMPTY = 4 };
+enum { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_FULL = 3, WAIT_ACC_EMPTY = 4, WAIT_SELFTEST = 9 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -47,14 +47,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // `code` in the global status word, raises the CTA's abort flag and returns; callers carry on to the
 // common tear-down so tensor memory is always released.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, long long max_cycles = WAIT_CYCLES) {
   if (mbar_try(bar, parity)) return;
   const long long t0 = clock64();
   int polls = 0;
   while (!mbar_try(bar, parity)) {
     if (*abort_flag) return;
     if ((++polls & 1023) == 0) {
-      if (*reinterpret_cast<volatile int*>(status) != 0 || clock64() - t0 > WAIT_CYCLES) {
+      if (*reinterpret_cast<volatile int*>(status) != 0 || clock64() - t0 > max_cycles) {
         atomicCAS(status, 0, code);
         *abort_flag = 1;
         return;
@@ -343,6 +343,19 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
+// One thread waits, with a short limit, on a barrier that nobody ever arrives at: the wait must give up by
+// itself, record its code and let the kernel end normally.
+__global__ void bounded_wait_probe_kernel(int* status, long long max_cycles) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait(smem_u32(&bar), 0, &abort_flag, status, WAIT_SELFTEST, max_cycles);
+  }
+}
+
 template <int BA, int BW, bool F32, int BN>
 cudaError_t launch_one(dim3 grid, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
                        const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw,
@@ -421,6 +434,15 @@ int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const
 }
 
 }  // namespace oq
+
+extern "C" int oq_selftest_bounded_wait(void* stream) {
+  int* status = oq::device_status_word();
+  if (!status) return oq::fail(OQ_ERR_CUDA, "oq_selftest_bounded_wait: cannot allocate the device status word");
+  oq::bounded_wait_probe_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(status, 2000000ll);   // ~1 ms
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return oq::cuda_fail(e, "oq_selftest_bounded_wait");
+  return OQ_OK;
+}
 
 extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
                           const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim,

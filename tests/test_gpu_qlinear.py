@@ -117,3 +117,19 @@ def test_strided_output_and_empty():
     with pytest.raises(B.OqError) as e:
         B.oq_qlinear(xq, xs, cb, wq, wr, B.oq_build_codebook(512, 4), d)
     assert e.value.code == 1
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A device-side wait whose barrier never completes must end by itself, leave the context usable and
+    show up in oq_device_status (nothing is hung or trapped to provoke it: the wait simply runs out)."""
+    import torch
+    assert B.oq_device_status() == 0
+    B.oq_selftest_bounded_wait()
+    assert B.oq_device_status() == 9          # code of the self-test wait; reading clears it
+    assert B.oq_device_status() == 0
+    d = 256
+    cb, rot = B.oq_build_codebook(d, 4), B.oq_make_rpbh(d, 128, 0)
+    xq, xs = B.oq_rotate_quantize_act(_dev(synth.activations(16, d, 1)), rot, cb)
+    wq, wr = B.oq_quantize_weights(_dev(synth.weights(16, d, 2)), rot, cb)
+    y = B.oq_qlinear(xq, xs, cb, wq, wr, cb, d)
+    assert torch.isfinite(y.float()).all() and B.oq_device_status() == 0
