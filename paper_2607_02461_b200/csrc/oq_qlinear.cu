@@ -143,17 +143,6 @@ __device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, 
   }
 }
 
-// Writes the four chunks of one (row, 32-coordinate half) into a K-major 128-byte-swizzled tile:
-// row r occupies 128 bytes; its 16-byte chunk c is stored at chunk position c ^ (r & 7).
-__device__ __forceinline__ void store_half(unsigned char* tile, int r, int half, const uint4 v[4]) {
-  unsigned char* row = tile + r * 128;
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int c = half * 4 + q;
-    *reinterpret_cast<uint4*>(row + ((c ^ (r & 7)) << 4)) = v[q];
-  }
-}
-
 // Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
@@ -203,13 +192,12 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
   if (warp == DECODE_THREADS / 32) {
     // ------------------------------- MMA issuer (one thread) -------------------------------
     if (lane == 0) {
-      uint32_t g = 0, lt = 0;
+      uint32_t st = 0, ph = 0, lt = 0;
       for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
         if (lt > 0) mbar_wait(accempty, (lt - 1) & 1, abort_flag, status, WAIT_ACC_EMPTY);   // epilogue drained TMEM
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        for (int kb = 0; kb < kblocks; ++kb, ++g) {
-          const uint32_t st = g % STAGES, use = g / STAGES;
-          mbar_wait(full0 + 8 * st, use & 1, abort_flag, status, WAIT_FULL);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          mbar_wait(full0 + 8 * st, ph, abort_flag, status, WAIT_FULL);
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_addr = smem_u32(smem + st * STAGE_BYTES);
           const uint64_t da0 = smem_desc(a_addr), da1 = smem_desc(a_addr + 128 * 128), db = smem_desc(a_addr + A_BYTES);
@@ -227,6 +215,7 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
           }
           // arrives on empty[st] once every MMA issued so far has finished reading shared memory
           asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(empty0 + 8 * st) : "memory");
+          if (++st == STAGES) { st = 0; ph ^= 1; }
         }
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(accfull) : "memory");
       }
@@ -236,50 +225,45 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
     const Tables ta = make_tables(cba), tw = make_tables(cbw);
     const int pitch_a = dim / 32 * BITS_A, pitch_w = dim / 32 * BITS_W;   // words per packed row
     const int row = tid >> 1, half = tid & 1;          // one (row, 32-coordinate half) of A and one of B per stage
-    uint32_t g = 0, lt = 0;
-    const uint32_t* a_src = nullptr;
-    const uint32_t* b_src = nullptr;
-    auto set_tile = [&](int tile) {
+    uint32_t st = 0, ph = 0, lt = 0;   // ring slot, phase parity of its current round, local tile count
+    bool first_round = true;           // nothing to wait for while the ring is filled for the first time
+    // byte offsets of this thread's four 16-byte chunks inside a K-major 128-byte-swizzled tile:
+    // row r occupies 128 bytes, its chunk c sits at chunk position c ^ (r & 7)
+    uint32_t toff[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) toff[q] = (uint32_t)row * 128u + ((uint32_t)((half * 4 + q) ^ (row & 7)) << 4);
+    // Packed words are fetched PF stages ahead of their decode (global/L2 latency under load is longer than
+    // one stage): ring of PF register sets, slot (stage index % PF).  dim % 128 == 0 makes the number of
+    // stages per tile even, so with PF = 2 the slot of a stage is the parity of its K block in every tile.
+    constexpr int PF = 2;
+    Raw<BITS_A> ra[PF];
+    Raw<BITS_W> rb[PF];
+    // position of the fetch stream: tile and K block of the next stage to fetch
+    int f_tile = blockIdx.x, f_kb = 0;
+    const uint32_t* fa = nullptr;
+    const uint32_t* fb = nullptr;
+    auto set_fetch_tile = [&](int tile) {
       const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
-      a_src = Aq + (size_t)min(n0 + row, n_tokens - 1) * pitch_a + half * BITS_A;   // rows past the end re-read the last
-      b_src = Wq + (size_t)min(i0 + row, m - 1) * pitch_w + half * BITS_W;          // row; their outputs are never stored
+      fa = Aq + (size_t)min(n0 + row, n_tokens - 1) * pitch_a + half * BITS_A;   // rows past the end re-read the last
+      fb = Wq + (size_t)min(i0 + row, m - 1) * pitch_w + half * BITS_W;          // row; their outputs are never stored
     };
-    Raw<BITS_A> ra;
-    Raw<BITS_W> rb;
-    if ((int)blockIdx.x < ntiles) {
-      set_tile(blockIdx.x);
-      ra = load_raw<BITS_A>(a_src);
-      rb = load_raw<BITS_W>(b_src);
-    }
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
-      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
-      for (int kb = 0; kb < kblocks; ++kb, ++g) {
-        const uint32_t st = g % STAGES, use = g / STAGES;
-        // fetch the next stage's packed words before decoding this one
-        Raw<BITS_A> na = ra;
-        Raw<BITS_W> nb = rb;
-        if (kb + 1 < kblocks) {
-          na = load_raw<BITS_A>(a_src + (size_t)(kb + 1) * 2 * BITS_A);
-          nb = load_raw<BITS_W>(b_src + (size_t)(kb + 1) * 2 * BITS_W);
-        } else if (tile + (int)gridDim.x < ntiles) {
-          set_tile(tile + gridDim.x);
-          na = load_raw<BITS_A>(a_src);
-          nb = load_raw<BITS_W>(b_src);
-        }
-        if (use > 0) mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort_flag, status, WAIT_EMPTY);
-        unsigned char* As = smem + st * STAGE_BYTES;
-        uint4 v[4];
-        decode32<BITS_A>(ra, ta, v);
-        store_half(As, row, half, v);
-        if (BN == BN_MAX || row < BN) {
-          decode32<BITS_W>(rb, tw, v);
-          store_half(As + A_BYTES, row, half, v);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
-        mbar_arrive(full0 + 8 * st);
-        ra = na;
-        rb = nb;
+    auto fetch_next = [&](Raw<BITS_A>& da, Raw<BITS_W>& db) {
+      if (f_tile >= ntiles) return;
+      da = load_raw<BITS_A>(fa);
+      db = load_raw<BITS_W>(fb);
+      fa += 2 * BITS_A;
+      fb += 2 * BITS_W;
+      if (++f_kb == kblocks) {
+        f_kb = 0;
+        f_tile += gridDim.x;
+        if (f_tile < ntiles) set_fetch_tile(f_tile);
       }
+    };
+    if (f_tile < ntiles) set_fetch_tile(f_tile);
+#pragma unroll
+    for (int i = 0; i < PF; ++i) fetch_next(ra[i], rb[i]);
+    auto epilogue = [&](int tile, uint32_t lt) {
+      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
       // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .., columns 128 (w / 4) ..; lane = one token row ----
       mbar_wait(accfull, lt & 1, abort_flag, status, WAIT_ACC_FULL);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -335,8 +319,34 @@ qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(accempty);   // this thread's TMEM reads are done: the next tile may overwrite the accumulators
+    };
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+     for (int kb = 0; kb < kblocks; kb += PF) {
+#pragma unroll
+      for (int u = 0; u < PF; ++u) {      // u = register set of this stage
+        const Raw<BITS_A> ca = ra[u];
+        const Raw<BITS_W> cb = rb[u];
+        fetch_next(ra[u], rb[u]);          // the stage PF ahead goes into the register set just freed
+        if (!first_round) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
+        unsigned char* As = smem + st * STAGE_BYTES;
+        uint4 v[4];
+        decode32<BITS_A>(ca, ta, v);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(As + toff[q]) = v[q];
+        if (BN == BN_MAX || row < BN) {
+          decode32<BITS_W>(cb, tw, v);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(As + A_BYTES + toff[q]) = v[q];
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+        mbar_arrive(full0 + 8 * st);
+        if (++st == STAGES) { st = 0; ph ^= 1; first_round = false; }
+      }
+     }
+     epilogue(tile, lt);
     }
   }
+
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 0)
