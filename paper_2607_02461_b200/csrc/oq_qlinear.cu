@@ -1,9 +1,10 @@
 // Codebook-decode GEMM:  Y[n][i] = s_n * r'_i * sum_k C_a[idxA[n][k]] * C_w[idxW[i][k]]
 // (the product W^' x^' of Sec. 4.3 with the magnitudes of Eq. 6 and Eq. 8 applied in the epilogue).
 //
-// Packed indices are fetched from global memory, decoded to bf16 levels with byte-permute table
-// look-ups, written into shared memory in the tensor core's K-major 128-byte-swizzled layout, and
-// contracted with tcgen05.mma (fp32 accumulators in tensor memory).
+// Packed indices are fetched from global memory into registers (one stage ahead), decoded to bf16 levels
+// with byte-permute table look-ups, written into shared memory in the tensor core's K-major
+// 128-byte-swizzled layout, and contracted with tcgen05.mma.cta_group::2 (fp32 accumulators in tensor
+// memory, two SMs per 256 x 256 tile).  Every device-side wait is bounded and reports to a status word.
 #include <cuda_bf16.h>
 
 #include "oq_internal.h"
@@ -12,16 +13,9 @@ namespace oq {
 
 namespace {
 
-constexpr int BM = 256;   // tokens per tile: two MMAs of M = 128, one accumulator each
-constexpr int BN_MAX = 256;   // features per tile (MMA N): 256, or 192 when that fills the last wave better
-constexpr int BK = 64;    // coordinates per stage: 64 bf16 = one 128-byte swizzled row
-constexpr int STAGES = 3;
-constexpr int DECODE_THREADS = 512;            // 16 warps decode and, after the last stage, run the epilogue
-constexpr int THREADS = DECODE_THREADS + 32;   // + one warp whose lane 0 issues the MMAs
-constexpr int TMEM_COLS = 512;                 // 2 accumulators x 256 fp32 columns
-constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN_MAX * BK * 2;
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr size_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int BK = 64;                  // coordinates per swizzle atom: 64 bf16 = one 128-byte swizzled row
+constexpr int DECODE_THREADS = 512;    // 16 decoding warps per CTA
+constexpr int TMEM_COLS = 512;         // two 128 x 256 fp32 accumulators per CTA
 constexpr long long WAIT_CYCLES = 4000000000ll;   // ~2 s: a wait that lasts longer reports and gives up
 
 enum { WAIT_EMPTY = 1, WAIT_FULL = 2, WAIT_ACC_FULL = 3, WAIT_ACC_EMPTY = 4, WAIT_SELFTEST = 9 };
@@ -30,9 +24,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -52,6 +43,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   const long long t0 = clock64();
   int polls = 0;
   while (!mbar_try(bar, parity)) {
+    __nanosleep(32);   // a waiting lane should not take issue slots from the warps it waits for
     if (*abort_flag) return;
     if ((++polls & 1023) == 0) {
       if (*reinterpret_cast<volatile int*>(status) != 0 || clock64() - t0 > max_cycles) {
@@ -147,210 +139,292 @@ __device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t idesc_for(int n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24); }
+// 32 lanes x 32 consecutive fp32 columns of tensor memory: thread i of the warp gets lane base + i.
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
 
-template <int BITS_A, int BITS_W, bool F32_OUT, int BN>
-__global__ void __launch_bounds__(THREADS, 1)
-qlinear_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm, int n_tokens,
-               const uint32_t* __restrict__ Wq, const __nv_bfloat16* __restrict__ w_norm, int m, int dim,
-               CodebookParams cba, CodebookParams cbw, void* __restrict__ Y, int ldy, int* status) {
+// ---------------------------------------------------------------------------------------------------------
+// Two-SM variant: a cluster of two CTAs computes one 256 x 256 tile with tcgen05.mma.cta_group::2.  Each
+// CTA decodes its own 128 token rows of A and its own 128 feature rows of B (the tensor cores of both SMs
+// read both halves of B, so every decoded byte of B is written once and used by 256 output rows), holds
+// 128 x 256 fp32 accumulators, double-buffered in its 512 TMEM columns, and stores its own 128 rows of Y.
+// CTA 0 of the pair issues the MMAs; "stage full" and "accumulator drained" arrivals from CTA 1 go to
+// CTA 0's barriers through the cluster address window, "stage free" and "accumulator ready" come back to
+// both CTAs with one multicast tcgen05.commit.  Dedicated epilogue warps overlap the epilogue of a tile
+// with the main loop of the next one.
+// ---------------------------------------------------------------------------------------------------------
+namespace pair {
+constexpr int PSTAGES = 3;
+constexpr int PBK = 2 * BK;                                            // 128 coordinates per stage: two swizzle atoms
+constexpr uint32_t ATOM_BYTES = 128 * BK * 2;                          // 128 rows x 128 bytes = 16 KB
+constexpr uint32_t PA_BYTES = 2 * ATOM_BYTES, PB_BYTES = 2 * ATOM_BYTES;
+constexpr uint32_t PSTAGE_BYTES = PA_BYTES + PB_BYTES;                 // 64 KB
+constexpr int EPI_THREADS = 128;
+constexpr int PTHREADS = DECODE_THREADS + EPI_THREADS + 32;   // 16 decode warps, 4 epilogue warps, 1 MMA warp
+constexpr size_t PSMEM_BYTES = PSTAGES * PSTAGE_BYTES + 1024 + 256;
+}  // namespace pair
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t local_bar, uint32_t rank) {
+  asm volatile(
+      "{\n .reg .b32 ra;\n mapa.shared::cluster.u32 ra, %0, %1;\n"
+      " mbarrier.arrive.shared::cluster.b64 _, [ra];\n}"
+      ::"r"(local_bar), "r"(rank) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait with cluster-scope acquire (the arrivals may come from the other CTA of the pair).
+__device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                  int code) {
+  if (mbar_try_cluster(bar, parity)) return;
+  const long long t0 = clock64();
+  int polls = 0;
+  while (!mbar_try_cluster(bar, parity)) {
+    if (*abort_flag) return;
+    if ((++polls & 1023) == 0) {
+      if (*reinterpret_cast<volatile int*>(status) != 0 || clock64() - t0 > WAIT_CYCLES) {
+        atomicCAS(status, 0, code);
+        *abort_flag = 1;
+        return;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void commit_multicast(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+// Decode loop of one thread of the two-SM kernel: the thread owns one (row, 32-coordinate half) of this CTA's
+// 128 rows of ONE operand (IS_A: activations, else weights) and, per 128-coordinate stage, decodes the two
+// 32-coordinate pieces that fall into the stage's two swizzle atoms.
+template <int BITS, bool IS_A>
+__device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ packed, int nrows, int dim, const Tables& t,
+                                                 unsigned char* smem, uint32_t full0, uint32_t empty0, int t2,
+                                                 uint32_t rank, int pair_id, int npairs, int ntiles, int tiles_n,
+                                                 int kblocks, volatile int* abort_flag, int* status) {
+  using namespace pair;
+  const int lane = threadIdx.x & 31;
+  const int row = t2 >> 1, half = t2 & 1;
+  const int pitch = dim / 32 * BITS;
+  constexpr int WPA = 2 * BITS;                       // words per 64 coordinates of one row
+  // swizzled chunk offsets inside a 128-row atom: row r occupies 128 bytes, chunk c sits at position c ^ (r & 7)
+  unsigned char* const tile0 = smem + (IS_A ? 0u : PA_BYTES) + (uint32_t)row * 128u;
+  uint32_t coff[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) coff[q] = (uint32_t)((half * 4 + q) ^ (row & 7)) << 4;
+  uint32_t st = 0, ph = 0;
+  bool first_round = true;
+  Raw<BITS> n0r, n1r;                                 // packed words of the NEXT stage
+  int f_tile = pair_id, f_kb = 0;
+  const uint32_t* fsrc = nullptr;
+  auto set_fetch_tile = [&](int tile) {
+    const int r0 = (IS_A ? (tile % tiles_n) : (tile / tiles_n)) * 256 + (int)rank * 128;
+    fsrc = packed + (size_t)min(r0 + row, nrows - 1) * pitch + half * BITS;   // rows past the end re-read the last row
+  };
+  auto fetch_next = [&]() {
+    if (f_tile >= ntiles) return;
+    n0r = load_raw<BITS>(fsrc);
+    n1r = load_raw<BITS>(fsrc + WPA);
+    fsrc += 2 * WPA;
+    if (++f_kb == kblocks) {
+      f_kb = 0;
+      f_tile += npairs;
+      if (f_tile < ntiles) set_fetch_tile(f_tile);
+    }
+  };
+  if (f_tile < ntiles) set_fetch_tile(f_tile);
+  fetch_next();
+  for (int tile = pair_id; tile < ntiles; tile += npairs) {
+    for (int kb = 0; kb < kblocks; ++kb) {
+      const Raw<BITS> c0 = n0r, c1 = n1r;
+      fetch_next();
+      if (!first_round) {
+        if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
+        __syncwarp();
+      }
+      unsigned char* Ss = tile0 + st * PSTAGE_BYTES;
+      uint4 v[4];
+      decode32<BITS>(c0, t, v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + coff[q]) = v[q];
+      decode32<BITS>(c1, t, v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ATOM_BYTES + coff[q]) = v[q];
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(full0 + 8 * st, 0);          // to CTA 0, where the MMAs are issued
+      if (++st == PSTAGES) { st = 0; ph ^= 1; first_round = false; }
+    }
+  }
+}
+
+template <int BITS_A, int BITS_W, bool F32_OUT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::PTHREADS, 1)
+qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm, int n_tokens,
+                    const uint32_t* __restrict__ Wq, const __nv_bfloat16* __restrict__ w_norm, int m, int dim,
+                    CodebookParams cba, CodebookParams cbw, void* __restrict__ Y, int ldy, int* status) {
+  using namespace pair;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + PSTAGES * PSTAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PSTAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
-  const uint32_t accfull = smem_u32(bars + 2 * STAGES), accempty = smem_u32(bars + 2 * STAGES + 1);
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + PSTAGES);
+  const uint32_t accfull0 = smem_u32(bars + 2 * PSTAGES), accempty0 = smem_u32(bars + 2 * PSTAGES + 2);
+  constexpr int MMA_WARP = (DECODE_THREADS + EPI_THREADS) / 32;
 
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full0 + 8 * s, DECODE_THREADS);   // every decoding thread arrives once per stage
-      mbar_init(empty0 + 8 * s, 1);               // tcgen05.commit arrives once the MMAs have read the stage
+    for (int s = 0; s < PSTAGES; ++s) {
+      mbar_init(full0 + 8 * s, 2 * (DECODE_THREADS / 32));   // one arrival per decoding warp of BOTH CTAs (used in CTA 0)
+      mbar_init(empty0 + 8 * s, 1);                          // multicast commit
     }
-    mbar_init(accfull, 1);                        // tcgen05.commit after the last stage of a tile
-    mbar_init(accempty, DECODE_THREADS);          // every epilogue thread arrives after reading its columns
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accfull0 + 8 * b, 1);                        // multicast commit
+      mbar_init(accempty0 + 8 * b, 2 * (EPI_THREADS / 32));  // epilogue warps of both CTAs (used in CTA 0)
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == MMA_WARP) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();     // barriers of both CTAs are initialised before anyone arrives remotely
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
 
-  const int kblocks = dim / BK;
-  const int tiles_n = (n_tokens + BM - 1) / BM, tiles_m = (m + BN - 1) / BN;
-  const int ntiles = tiles_n * tiles_m;   // token tiles vary fastest: CTAs running together share weight rows
+  const int kblocks = dim / PBK;
+  const int tiles_n = (n_tokens + 255) / 256;
+  const int ntiles = tiles_n * ((m + 255) / 256);
+  const int npairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
 
-  if (warp == DECODE_THREADS / 32) {
-    // ------------------------------- MMA issuer (one thread) -------------------------------
-    if (lane == 0) {
+  if (warp == MMA_WARP) {
+    // ------------------------------- MMA issuer: one thread of CTA 0 -------------------------------
+    if (rank == 0 && lane == 0) {
       uint32_t st = 0, ph = 0, lt = 0;
-      for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
-        if (lt > 0) mbar_wait(accempty, (lt - 1) & 1, abort_flag, status, WAIT_ACC_EMPTY);   // epilogue drained TMEM
+      constexpr uint32_t IDESC2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
+        const uint32_t buf = lt & 1;
+        if (lt >= 2) mbar_wait_cluster(accempty0 + 8 * buf, ((lt >> 1) - 1) & 1, abort_flag, status, WAIT_ACC_EMPTY);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         for (int kb = 0; kb < kblocks; ++kb) {
-          mbar_wait(full0 + 8 * st, ph, abort_flag, status, WAIT_FULL);
+          mbar_wait_cluster(full0 + 8 * st, ph, abort_flag, status, WAIT_FULL);
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = smem_u32(smem + st * STAGE_BYTES);
-          const uint64_t da0 = smem_desc(a_addr), da1 = smem_desc(a_addr + 128 * 128), db = smem_desc(a_addr + A_BYTES);
+          const uint32_t a_addr = smem_u32(smem + st * PSTAGE_BYTES);
 #pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4) {
+          for (int k4 = 0; k4 < PBK / 16; ++k4) {
+            // K step k4: swizzle atom k4 / 4, 32 bytes per step inside the atom
+            const uint64_t da = smem_desc(a_addr + (k4 >> 2) * ATOM_BYTES) + 2 * (k4 & 3);
+            const uint64_t db = smem_desc(a_addr + PA_BYTES + (k4 >> 2) * ATOM_BYTES) + 2 * (k4 & 3);
             const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
             asm volatile(
                 "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-                " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                ::"r"(tmem), "l"(da0 + 2 * k4), "l"(db + 2 * k4), "r"(idesc_for(BN)), "r"(acc) : "memory");
-            asm volatile(
-                "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-                " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                ::"r"(tmem + BN), "l"(da1 + 2 * k4), "l"(db + 2 * k4), "r"(idesc_for(BN)), "r"(acc) : "memory");
+                " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+                ::"r"(tmem + buf * 256), "l"(da), "l"(db), "r"(IDESC2), "r"(acc) : "memory");
           }
-          // arrives on empty[st] once every MMA issued so far has finished reading shared memory
-          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(empty0 + 8 * st) : "memory");
-          if (++st == STAGES) { st = 0; ph ^= 1; }
+          commit_multicast(empty0 + 8 * st);       // both CTAs may refill the stage once these MMAs have read it
+          if (++st == PSTAGES) { st = 0; ph ^= 1; }
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(accfull) : "memory");
+        commit_multicast(accfull0 + 8 * buf);      // both CTAs' epilogue warps may read accumulator `buf`
       }
     }
-  } else {
-    // ------------------- decoders (all 16 warps), then the epilogue of the tile -------------------
-    const Tables ta = make_tables(cba), tw = make_tables(cbw);
-    const int pitch_a = dim / 32 * BITS_A, pitch_w = dim / 32 * BITS_W;   // words per packed row
-    const int row = tid >> 1, half = tid & 1;          // one (row, 32-coordinate half) of A and one of B per stage
-    uint32_t st = 0, ph = 0, lt = 0;   // ring slot, phase parity of its current round, local tile count
-    bool first_round = true;           // nothing to wait for while the ring is filled for the first time
-    // byte offsets of this thread's four 16-byte chunks inside a K-major 128-byte-swizzled tile:
-    // row r occupies 128 bytes, its chunk c sits at chunk position c ^ (r & 7)
-    uint32_t toff[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) toff[q] = (uint32_t)row * 128u + ((uint32_t)((half * 4 + q) ^ (row & 7)) << 4);
-    // Packed words are fetched PF stages ahead of their decode (global/L2 latency under load is longer than
-    // one stage): ring of PF register sets, slot (stage index % PF).  dim % 128 == 0 makes the number of
-    // stages per tile even, so with PF = 2 the slot of a stage is the parity of its K block in every tile.
-    constexpr int PF = 2;
-    Raw<BITS_A> ra[PF];
-    Raw<BITS_W> rb[PF];
-    // position of the fetch stream: tile and K block of the next stage to fetch
-    int f_tile = blockIdx.x, f_kb = 0;
-    const uint32_t* fa = nullptr;
-    const uint32_t* fb = nullptr;
-    auto set_fetch_tile = [&](int tile) {
-      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
-      fa = Aq + (size_t)min(n0 + row, n_tokens - 1) * pitch_a + half * BITS_A;   // rows past the end re-read the last
-      fb = Wq + (size_t)min(i0 + row, m - 1) * pitch_w + half * BITS_W;          // row; their outputs are never stored
-    };
-    auto fetch_next = [&](Raw<BITS_A>& da, Raw<BITS_W>& db) {
-      if (f_tile >= ntiles) return;
-      da = load_raw<BITS_A>(fa);
-      db = load_raw<BITS_W>(fb);
-      fa += 2 * BITS_A;
-      fb += 2 * BITS_W;
-      if (++f_kb == kblocks) {
-        f_kb = 0;
-        f_tile += gridDim.x;
-        if (f_tile < ntiles) set_fetch_tile(f_tile);
-      }
-    };
-    if (f_tile < ntiles) set_fetch_tile(f_tile);
-#pragma unroll
-    for (int i = 0; i < PF; ++i) fetch_next(ra[i], rb[i]);
-    auto epilogue = [&](int tile, uint32_t lt) {
-      const int n0 = (tile % tiles_n) * BM, i0 = (tile / tiles_n) * BN;
-      // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .., columns 128 (w / 4) ..; lane = one token row ----
-      mbar_wait(accfull, lt & 1, abort_flag, status, WAIT_ACC_FULL);
+  } else if (warp >= DECODE_THREADS / 32) {
+    // ------------------------------- epilogue warps (4 per CTA) -------------------------------
+    const int q = warp & 3;                          // TMEM lane quarter of this warp
+    uint32_t lt = 0;
+    for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
+      const uint32_t buf = lt & 1;
+      const int n0 = (tile % tiles_n) * 256 + (int)rank * 128, i0 = (tile / tiles_n) * 256;
+      if (lane == 0) mbar_wait(accfull0 + 8 * buf, (lt >> 1) & 1, abort_flag, status, WAIT_ACC_FULL);
+      __syncwarp();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      __syncwarp();   // the per-thread wait loops may leave the warp diverged; tcgen05.ld is warp-collective
-      {
-        const int cg = warp >> 2;                        // column group: accumulator cg / 2, feature half cg % 2
-        const int trow = n0 + (cg >> 1) * 128 + (warp & 3) * 32 + lane;
-        const float s = trow < n_tokens ? a_norm[trow] : 0.f;
+      const int trow = n0 + q * 32 + lane;
+      const float s = trow < n_tokens ? a_norm[trow] : 0.f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 64; ++c) {
-          const int fcol = (cg & 1) * (BN / 2) + c * 32;   // feature offset inside the tile
-          uint32_t r[32];
-          const uint32_t taddr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((cg >> 1) * BN + fcol);
-          asm volatile(
-              "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-              "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-                "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-                "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-                "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-              : "r"(taddr)
-              : "memory");
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (trow < n_tokens) {
+      for (int c = 0; c < 8; ++c) {
+        uint32_t r[32];
+        tmem_load32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c * 32), r);
+        if (trow < n_tokens) {
 #pragma unroll
-            for (int g8 = 0; g8 < 4; ++g8) {   // 8 features per group
-              const int i = i0 + fcol + g8 * 8;
-              if (i < m) {
-                const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));   // 8 bf16 row norms
-                const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
-                float y[8];
+          for (int g8 = 0; g8 < 4; ++g8) {
+            const int i = i0 + c * 32 + g8 * 8;
+            if (i < m) {
+              const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));
+              const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
+              float y[8];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  y[2 * j] = (__uint_as_float(r[g8 * 8 + 2 * j]) * s) * __uint_as_float(rw[j] << 16);
-                  y[2 * j + 1] = (__uint_as_float(r[g8 * 8 + 2 * j + 1]) * s) * __uint_as_float(rw[j] & 0xFFFF0000u);
-                }
-                if (F32_OUT) {
-                  float* dst = reinterpret_cast<float*>(Y) + (size_t)trow * ldy + i;
-                  *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
-                  *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
-                } else {
-                  __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
-                  __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
-                  uint4 pk;
-                  pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                  pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                  *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(Y) + (size_t)trow * ldy + i) = pk;
-                }
+              for (int jj = 0; jj < 4; ++jj) {
+                y[2 * jj] = (__uint_as_float(r[g8 * 8 + 2 * jj]) * s) * __uint_as_float(rw[jj] << 16);
+                y[2 * jj + 1] = (__uint_as_float(r[g8 * 8 + 2 * jj + 1]) * s) * __uint_as_float(rw[jj] & 0xFFFF0000u);
+              }
+              if (F32_OUT) {
+                float* dst = reinterpret_cast<float*>(Y) + (size_t)trow * ldy + i;
+                *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
+                *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
+              } else {
+                __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
+                __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
+                uint4 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(Y) + (size_t)trow * ldy + i) = pk;
               }
             }
           }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(accempty);   // this thread's TMEM reads are done: the next tile may overwrite the accumulators
-    };
-    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
-     for (int kb = 0; kb < kblocks; kb += PF) {
-#pragma unroll
-      for (int u = 0; u < PF; ++u) {      // u = register set of this stage
-        const Raw<BITS_A> ca = ra[u];
-        const Raw<BITS_W> cb = rb[u];
-        fetch_next(ra[u], rb[u]);          // the stage PF ahead goes into the register set just freed
-        if (!first_round) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
-        unsigned char* As = smem + st * STAGE_BYTES;
-        uint4 v[4];
-        decode32<BITS_A>(ca, ta, v);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(As + toff[q]) = v[q];
-        if (BN == BN_MAX || row < BN) {
-          decode32<BITS_W>(cb, tw, v);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(As + A_BYTES + toff[q]) = v[q];
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
-        mbar_arrive(full0 + 8 * st);
-        if (++st == STAGES) { st = 0; ph ^= 1; first_round = false; }
-      }
-     }
-     epilogue(tile, lt);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(accempty0 + 8 * buf, 0);   // CTA 0 may let the MMAs overwrite `buf`
+    }
+  } else {
+    // ------------------------------- decoders (16 warps per CTA) -------------------------------
+    // threads 0-255: this CTA's 128 rows of A; threads 256-511: its 128 rows of B
+    if (tid < 256) {
+      const Tables ta = make_tables(cba);
+      pair_decode_loop<BITS_A, true>(Aq, n_tokens, dim, ta, smem, full0, empty0, tid, rank, pair_id, npairs, ntiles,
+                                     tiles_n, kblocks, abort_flag, status);
+    } else {
+      const Tables tw = make_tables(cbw);
+      pair_decode_loop<BITS_W, false>(Wq, m, dim, tw, smem, full0, empty0, tid - 256, rank, pair_id, npairs, ntiles,
+                                      tiles_n, kblocks, abort_flag, status);
     }
   }
-
+  __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  cluster_sync_all();     // neither CTA leaves (or frees TMEM) while the other may still signal it or read its tiles
+  if (warp == MMA_WARP) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
 // One thread waits, with a short limit, on a barrier that nobody ever arrives at: the wait must give up by
@@ -366,29 +440,42 @@ __global__ void bounded_wait_probe_kernel(int* status, long long max_cycles) {
   }
 }
 
-template <int BA, int BW, bool F32, int BN>
-cudaError_t launch_one(dim3 grid, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
-                       const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw,
-                       void* Y, int ldy, int* status) {
-  auto k = qlinear_kernel<BA, BW, F32, BN>;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+template <int BA, int BW, bool F32>
+cudaError_t launch_pair(int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
+                        const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw,
+                        void* Y, int ldy, int* status) {
+  auto k = qlinear_pair_kernel<BA, BW, F32>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pair::PSMEM_BYTES);
   if (e != cudaSuccess) return e;
-  k<<<grid, THREADS, SMEM_BYTES, st>>>(Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
+  const int ntiles = ((n + 255) / 256) * ((m + 255) / 256);
+  // persistent grid: as many pairs as can be resident at once (SM pairs must sit in one cluster-capable group,
+  // so this can be fewer than sms / 2)
+  static int max_pairs[64] = {0};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && max_pairs[dev] == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sms / 2 * 2);
+    cfg.blockDim = dim3(pair::PTHREADS);
+    cfg.dynamicSmemBytes = pair::PSMEM_BYTES;
+    int nclusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&nclusters, k, &cfg);
+    if (e != cudaSuccess) return e;
+    max_pairs[dev] = nclusters > 0 ? nclusters : 1;
+  }
+  int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev] : sms / 2;
+  if (pairs > sms / 2) pairs = sms / 2;
+  if (pairs > ntiles) pairs = ntiles;
+  k<<<2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st>>>(Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
   return cudaGetLastError();
 }
 
 template <int BA, int BW>
-int launch_bits(bool f32, int bn, dim3 grid, cudaStream_t st, const uint32_t* Aq, const float* an, int n,
-                const uint32_t* Wq, const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca,
-                const CodebookParams& cw, void* Y, int ldy, int* status) {
-  cudaError_t e;
-  if (f32) {
-    e = bn == 256 ? launch_one<BA, BW, true, 256>(grid, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status)
-                  : launch_one<BA, BW, true, 192>(grid, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
-  } else {
-    e = bn == 256 ? launch_one<BA, BW, false, 256>(grid, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status)
-                  : launch_one<BA, BW, false, 192>(grid, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
-  }
+int launch_bits(bool f32, int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
+                const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw, void* Y,
+                int ldy, int* status) {
+  const cudaError_t e = f32 ? launch_pair<BA, BW, true>(sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status)
+                            : launch_pair<BA, BW, false>(sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
   if (e != cudaSuccess) return cuda_fail(e, "oq_qlinear launch");
   return OQ_OK;
 }
@@ -423,21 +510,13 @@ int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const
   cudaGetDevice(&dev);
   cudaError_t ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (ce != cudaSuccess) return cuda_fail(ce, "cudaDeviceGetAttribute");
-  // Tile width: 256 features, or 192 when the narrower tiles leave less of the last wave empty
-  // (a 192-wide tile does 3/4 of the work at roughly 9/10 of the efficiency).
-  const int tiles_tok = (n_tokens + BM - 1) / BM;
-  const int t256 = tiles_tok * ((m + 255) / 256), t192 = tiles_tok * ((m + 191) / 192);
-  const double cost256 = (double)((t256 + sms - 1) / sms), cost192 = 0.85 * (double)((t192 + sms - 1) / sms);
-  const int bn = cost192 < cost256 ? 192 : 256;
-  const int ntiles = bn == 256 ? t256 : t192;
-  dim3 grid(ntiles < sms ? ntiles : sms);   // persistent: one CTA per SM walks the tiles
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const uint32_t* A = reinterpret_cast<const uint32_t*>(Xq_idx);
   const uint32_t* W = reinterpret_cast<const uint32_t*>(Wq_idx);
   const __nv_bfloat16* wn = reinterpret_cast<const __nv_bfloat16*>(Wq_norm_bf16);
   const bool f32 = y_dtype == OQ_F32;
 #define OQ_CASE(a, w) \
-  if (ba == a && bw == w) return launch_bits<a, w>(f32, bn, grid, st, A, Xq_norm, n_tokens, W, wn, m, dim, ca, cw, Y, ldy, status);
+  if (ba == a && bw == w) return launch_bits<a, w>(f32, sms, st, A, Xq_norm, n_tokens, W, wn, m, dim, ca, cw, Y, ldy, status);
   OQ_CASE(4, 4) OQ_CASE(3, 3) OQ_CASE(4, 2) OQ_CASE(3, 2) OQ_CASE(4, 3) OQ_CASE(2, 2) OQ_CASE(3, 4) OQ_CASE(2, 4) OQ_CASE(2, 3)
 #undef OQ_CASE
   return fail(OQ_ERR_UNSUPPORTED, "oq_qlinear: unsupported bit-width pair");
