@@ -313,14 +313,14 @@ def run_ours(args):
                    "layers": [f"{l['name']} {l['d']}->{l['m']}" for l in L], "bits_w": bw, "bits_a": ba,
                    "rpbh_block": block, "parallelism": f"token-sharded replicas x{world}, no collective",
                    "l2": "256 MiB buffer written between steps, outside the event-timed spans"},
-        "roofline": {"bound": "tensor", "kernel": "qlinear_kernel", "achieved": gemm_tf,
+        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel", "achieved": gemm_tf,
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / pk["bf16_tflops"],
                      "traffic": (traffic or {}).get("qlinear_bytes_per_step"),
                      "peak_source": f"{pk['source']} burst (sustained {pk['bf16_tflops_sustained']})",
                      "frac_of_nominal_2250": gemm_tf / 2250.0,
                      "per_layer_tflops": {l["name"]: 2 * tokens * l["m"] * l["d"] / (gemm_ms[i] * 1e-3) / 1e12
                                           for i, l in enumerate(L)}},
-        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
+        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq_fast_kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
                                      "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
                                      "traffic": (traffic or {}).get("rq_bytes_per_step"),
                                      "algorithmic_bytes_per_step": rq_b, "frac_of_nominal_8000": rq_gbs / 8000.0,
