@@ -149,7 +149,7 @@ static bool plan_fast(int dim, int block, const oq_codebook* cb, FastPlan* plan)
   plan->ctas_per_sm = ctas;
   plan->threads = RQ_MAX_THREADS / ctas;
   plan->smem = smem_of(T);
-  // copying threads: enough whole warps that each handles at most rq_words_per_thread(T) words per row
+  // copying threads: enough whole warps that each handles rq_words_per_thread(T) consecutive words per row
   const int maxw = rq_words_per_thread(T);
   int ncopy = ((dim / 2 + maxw - 1) / maxw + 31) / 32 * 32;
   if (ncopy > plan->threads) return false;

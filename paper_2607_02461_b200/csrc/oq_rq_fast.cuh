@@ -202,7 +202,9 @@ __device__ __forceinline__ void pack32(const float* z, float kappa, const Poly2<
 }
 
 constexpr int RQ_MAX_THREADS = 512;
-__host__ __device__ constexpr int rq_words_per_thread(int T) { return T >= 16 ? 3 : T == 8 ? 6 : 14; }
+// consecutive 32-bit words of a row handled by one copying thread; odd, so that a warp's accesses at this
+// stride fall into distinct shared-memory banks
+__host__ __device__ constexpr int rq_words_per_thread(int T) { return T >= 16 ? 3 : T == 8 ? 7 : 15; }
 
 template <int H, int T, int BITS>
 __global__ void __launch_bounds__(RQ_MAX_THREADS, 1) rq_fast_kernel(const RqFastParams p) {
@@ -223,30 +225,32 @@ __global__ void __launch_bounds__(RQ_MAX_THREADS, 1) rq_fast_kernel(const RqFast
 
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, nwarps = nthr >> 5;
   const int wd = p.dim / 2;
-  // the first p.ncopy threads (whole warps) move and pre-process the rows, MAXW words each at most
-  const int ncopy = p.ncopy;
-  const bool copier = tid < ncopy;
-  const int nw_thr = copier ? (wd - tid + ncopy - 1) / ncopy : 0;
+  // the first p.ncopy threads (whole warps) move and pre-process the rows: thread t owns the MAXW consecutive
+  // words [t MAXW, (t+1) MAXW) of every row (immediate offsets, no per-word address arithmetic)
+  const int w0 = tid * MAXW;
+  const bool copier = tid < p.ncopy && w0 < wd;
+  const int nw_thr = copier ? min(MAXW, wd - w0) : 0;
 
   uint32_t mask[MAXW];
 #pragma unroll
-  for (int q = 0; q < MAXW; ++q) mask[q] = q < nw_thr ? __ldg(p.srcmask + tid + q * ncopy) : 0u;
+  for (int q = 0; q < MAXW; ++q) mask[q] = q < nw_thr ? __ldg(p.srcmask + w0 + q) : 0u;
 
   // Asynchronous copy of one group of T rows into buffer `buf` (4 bytes per lane per instruction, no
   // registers held while the data is in flight).
   auto issue_group = [&](int grp, int buf) {
     if (!copier) return;
     const int row0 = grp * T;
-    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(rowbuf0 + buf * T * pitch_w + tid);
+    uint32_t dst = (uint32_t)__cvta_generic_to_shared(rowbuf0 + buf * T * pitch_w + w0);
+    const uint32_t* src = p.X + (size_t)row0 * p.ldw + w0;
+    const int last = p.rows - 1 - row0;              // rows past the end re-read the last row
 #pragma unroll
     for (int r = 0; r < T; ++r) {
-      const int row = min(row0 + r, p.rows - 1);
-      const uint32_t* src = p.X + (size_t)row * p.ldw + tid;
-      const uint32_t dst = dst0 + (uint32_t)(r * pitch_w) * 4u;
+      const uint32_t* s = src + (size_t)min(r, last) * p.ldw;
 #pragma unroll
       for (int q = 0; q < MAXW; ++q)
         if (q < nw_thr)
-          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + (uint32_t)(q * ncopy) * 4u), "l"(src + q * ncopy) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst + 4u * q), "l"(s + q) : "memory");
+      dst += (uint32_t)pitch_w * 4u;
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
@@ -277,19 +281,20 @@ __global__ void __launch_bounds__(RQ_MAX_THREADS, 1) rq_fast_kernel(const RqFast
     for (int r = 0; r < T; ++r) ssq[r] = 0.f;
     if (copier) {
 #pragma unroll
-      for (int r = 0; r < T; ++r) {
-        uint32_t* rw = rowbuf + r * pitch_w + tid;
+      uint32_t* rw = rowbuf + w0;
+#pragma unroll
+      for (int r = 0; r < T; ++r, rw += pitch_w) {
         uint32_t w[MAXW];
 #pragma unroll
         for (int q = 0; q < MAXW; ++q)
-          if (q < nw_thr) w[q] = rw[q * ncopy];
+          if (q < nw_thr) w[q] = rw[q];
         unsigned long long acc2 = 0ull;
 #pragma unroll
         for (int q = 0; q < MAXW; ++q)
           if (q < nw_thr) {
             const unsigned long long x2 = pack2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xFFFF0000u));
             acc2 = fma2(x2, x2, acc2);
-            if (mask[q]) rw[q * ncopy] = w[q] ^ mask[q];
+            rw[q] = w[q] ^ mask[q];
           }
         float a0, a1;
         unpack2(acc2, a0, a1);
