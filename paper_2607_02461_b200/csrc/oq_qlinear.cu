@@ -103,6 +103,25 @@ __device__ __forceinline__ Raw<BITS> load_raw(const uint32_t* __restrict__ src) 
   return r;
 }
 
+// The 2 * BITS contiguous words of 64 coordinates of one row, as two 32-coordinate pieces.
+template <int BITS>
+__device__ __forceinline__ void load_raw64(const uint32_t* __restrict__ src, Raw<BITS>& a, Raw<BITS>& b) {
+  if (BITS == 4) {          // 32 bytes, 16-byte aligned
+    a = load_raw<BITS>(src);
+    b = load_raw<BITS>(src + 4);
+  } else if (BITS == 3) {   // 24 bytes, 8-byte aligned
+    const uint2 v0 = __ldg(reinterpret_cast<const uint2*>(src));
+    const uint2 v1 = __ldg(reinterpret_cast<const uint2*>(src) + 1);
+    const uint2 v2 = __ldg(reinterpret_cast<const uint2*>(src) + 2);
+    a.w[0] = v0.x; a.w[1] = v0.y; a.w[BITS - 1] = v1.x;
+    b.w[0] = v1.y; b.w[1] = v2.x; b.w[BITS - 1] = v2.y;
+  } else {                  // 16 bytes, 16-byte aligned
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+    a.w[0] = v.x; a.w[1] = v.y;
+    b.w[0] = v.z; b.w[1] = v.w;
+  }
+}
+
 template <int BITS>
 __device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, uint4 out[4]) {
   if (BITS == 4) {
@@ -119,12 +138,26 @@ __device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, 
   } else {
     const uint32_t mw[2] = {raw.w[0], raw.w[BITS == 3 ? 1 : 0]};
     const uint32_t s = raw.w[BITS - 1];
+    // byte-permute selectors of the 8 groups of 4 coordinates: the permute reads only the low 16 bits of a
+    // selector, so one mask serves two groups (the second after a shift by 16)
+    uint32_t selv[8];
+    if (BITS == 3) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const uint32_t e = mw[u] & 0x33333333u, o = (mw[u] >> 2) & 0x33333333u;
+        selv[4 * u] = e; selv[4 * u + 1] = o; selv[4 * u + 2] = e >> 16; selv[4 * u + 3] = o >> 16;
+      }
+    } else {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t e = (mw[0] >> g) & 0x11111111u;
+        selv[g] = e; selv[4 + g] = e >> 16;
+      }
+    }
     uint32_t r[16];
 #pragma unroll
     for (int G = 0; G < 8; ++G) {
-      uint32_t sel;
-      if (BITS == 3) sel = (mw[G >> 2] >> (2 * (G & 1) + 16 * ((G >> 1) & 1))) & 0x3333u;
-      else sel = (mw[0] >> ((G & 3) + 16 * (G >> 2))) & 0x1111u;
+      const uint32_t sel = selv[G];
       const uint32_t lo = prmt(t.lo0, t.lo0, sel);
       const uint32_t hi = prmt(t.hi0, t.hi0, sel) ^ ((s << G) & 0x80808080u);
       r[2 * G] = prmt(lo, hi, 0x5140u);
@@ -228,14 +261,22 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
                                                  int kblocks, volatile int* abort_flag, int* status) {
   using namespace pair;
   const int lane = threadIdx.x & 31;
-  const int row = t2 >> 1, half = t2 & 1;
+  // Two ways to split a stage's 128 rows x 128 coordinates among 256 threads:
+  //  * 4-bit operands: thread = (row t2/2, 32-coordinate half t2%2) of BOTH 64-coordinate swizzle atoms: one
+  //    16-byte load per piece, adjacent lanes read adjacent 16 bytes;
+  //  * 3- and 2-bit operands: thread = (row t2%128, atom t2/128), 64 contiguous coordinates: 24 / 16 bytes,
+  //    8- / 16-byte aligned, instead of 12- / 8-byte pieces.
+  // Inside an atom row r occupies 128 bytes and its 16-byte chunk c sits at position c ^ (r & 7); both
+  // mappings give the 8 lanes of a quarter warp 8 different chunk positions, i.e. all 32 banks.
+  constexpr bool CONTIG = BITS != 4;
+  const int row = CONTIG ? (t2 & 127) : (t2 >> 1);
+  const int sub = CONTIG ? (t2 >> 7) : (t2 & 1);      // atom (CONTIG) or half of each atom
   const int pitch = dim / 32 * BITS;
   constexpr int WPA = 2 * BITS;                       // words per 64 coordinates of one row
-  // swizzled chunk offsets inside a 128-row atom: row r occupies 128 bytes, chunk c sits at position c ^ (r & 7)
-  unsigned char* const tile0 = smem + (IS_A ? 0u : PA_BYTES) + (uint32_t)row * 128u;
-  uint32_t coff[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) coff[q] = (uint32_t)((half * 4 + q) ^ (row & 7)) << 4;
+  unsigned char* const tile0 = smem + (IS_A ? 0u : PA_BYTES) + (uint32_t)row * 128u + (CONTIG ? (uint32_t)sub * ATOM_BYTES : 0u);
+  const uint32_t rx = (uint32_t)(row & 7) << 4;
+  const uint32_t c0b = CONTIG ? 0u : (uint32_t)sub * 64u;          // first chunk (in bytes) of the first piece
+  const uint32_t second = CONTIG ? 64u : ATOM_BYTES;                // where the second piece goes relative to it
   uint32_t st = 0, ph = 0;
   bool first_round = true;
   Raw<BITS> n0r, n1r;                                 // packed words of the NEXT stage
@@ -243,12 +284,16 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
   const uint32_t* fsrc = nullptr;
   auto set_fetch_tile = [&](int tile) {
     const int r0 = (IS_A ? (tile % tiles_n) : (tile / tiles_n)) * 256 + (int)rank * 128;
-    fsrc = packed + (size_t)min(r0 + row, nrows - 1) * pitch + half * BITS;   // rows past the end re-read the last row
+    fsrc = packed + (size_t)min(r0 + row, nrows - 1) * pitch + sub * (CONTIG ? WPA : BITS);   // rows past the end re-read the last
   };
   auto fetch_next = [&]() {
     if (f_tile >= ntiles) return;
-    n0r = load_raw<BITS>(fsrc);
-    n1r = load_raw<BITS>(fsrc + WPA);
+    if (CONTIG) {
+      load_raw64<BITS>(fsrc, n0r, n1r);
+    } else {
+      n0r = load_raw<BITS>(fsrc);
+      n1r = load_raw<BITS>(fsrc + WPA);
+    }
     fsrc += 2 * WPA;
     if (++f_kb == kblocks) {
       f_kb = 0;
@@ -270,10 +315,15 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
       uint4 v[4];
       decode32<BITS>(c0, t, v);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + coff[q]) = v[q];
+      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ((c0b + ((uint32_t)q << 4)) ^ rx)) = v[q];
       decode32<BITS>(c1, t, v);
+      if (CONTIG) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ATOM_BYTES + coff[q]) = v[q];
+        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ((second + ((uint32_t)q << 4)) ^ rx)) = v[q];
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + second + ((c0b + ((uint32_t)q << 4)) ^ rx)) = v[q];
+      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(full0 + 8 * st, 0);          // to CTA 0, where the MMAs are issued

@@ -280,7 +280,6 @@ __global__ void __launch_bounds__(RQ_MAX_THREADS, 1) rq_fast_kernel(const RqFast
 #pragma unroll
     for (int r = 0; r < T; ++r) ssq[r] = 0.f;
     if (copier) {
-#pragma unroll
       uint32_t* rw = rowbuf + w0;
 #pragma unroll
       for (int r = 0; r < T; ++r, rw += pitch_w) {
