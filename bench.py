@@ -194,7 +194,10 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    oqbuild.build()
+    if rank == 0:
+        oqbuild.build()          # no-op when liboq.so is newer than its sources
+    if world > 1:
+        dist.barrier()           # the other ranks load the library only after rank 0 has made sure it is built
     B.lib()
 
     tokens, layers, bw, ba, block = WORKLOADS[args.workload]
