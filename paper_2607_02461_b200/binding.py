@@ -49,6 +49,7 @@ def lib():
             "oq_linear_forward_host": (i, [vp, i, i, vp, vp, vp, vp, i, vp, vp, vp, sz, vp]),
             "oq_device_status": (i, [C.POINTER(i)]),
             "oq_selftest_bounded_wait": (i, [vp]),
+            "oq_debug_select_rq_kernel": (i, [i]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
         for name, (res, args) in sig.items():
@@ -214,6 +215,10 @@ def oq_device_status():
 
 def oq_selftest_bounded_wait():
     _check(lib().oq_selftest_bounded_wait(_stream()))
+
+
+def oq_debug_select_rq_kernel(which):
+    _check(lib().oq_debug_select_rq_kernel(int(which)))
 
 
 def oq_version():

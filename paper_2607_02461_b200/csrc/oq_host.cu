@@ -211,17 +211,23 @@ int ensure_device_tables(const oq_rpbh* rc) {
   if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
   e = cudaMemcpy(r->d_gather, g.data(), sizeof(uint32_t) * r->dim, cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
-  std::vector<uint32_t> off(r->dim), mask((r->dim + 1) / 2, 0u);
+  std::vector<uint32_t> off(r->dim), mask((r->dim + 1) / 2, 0u), pmask((r->dim + 1) / 2, 0u);
   for (int k = 0; k < r->dim; ++k) {
     off[k] = 2u * (uint32_t)r->perm[k];
-    if (r->signs[k] < 0) mask[r->perm[k] >> 1] |= (r->perm[k] & 1) ? 0x80000000u : 0x00008000u;
+    if (r->signs[k] < 0) {
+      mask[r->perm[k] >> 1] |= (r->perm[k] & 1) ? 0x80000000u : 0x00008000u;
+      pmask[k >> 1] |= (k & 1) ? 0x80000000u : 0x00008000u;
+    }
   }
   e = cudaMalloc(&r->d_offset, sizeof(uint32_t) * off.size());
   if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
   e = cudaMalloc(&r->d_srcmask, sizeof(uint32_t) * mask.size());
   if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
+  e = cudaMalloc(&r->d_posmask, sizeof(uint32_t) * pmask.size());
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
   e = cudaMemcpy(r->d_offset, off.data(), sizeof(uint32_t) * off.size(), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(r->d_srcmask, mask.data(), sizeof(uint32_t) * mask.size(), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(r->d_posmask, pmask.data(), sizeof(uint32_t) * pmask.size(), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
   r->device = dev;
   return OQ_OK;
@@ -358,6 +364,7 @@ void oq_rpbh_destroy(oq_rpbh* r) {
   if (r->d_gather) cudaFree(r->d_gather);
   if (r->d_offset) cudaFree(r->d_offset);
   if (r->d_srcmask) cudaFree(r->d_srcmask);
+  if (r->d_posmask) cudaFree(r->d_posmask);
   delete r;
 }
 

@@ -41,6 +41,8 @@ struct oq_rpbh {
   uint32_t* d_offset = nullptr;  // [dim] byte offset 2 * perm[k] of the source element of rotated position k
   uint32_t* d_srcmask = nullptr; // [dim/2] bf16x2 sign-bit masks indexed by SOURCE position: 0x8000 where the
                                  // element moves to a position whose sign is -1
+  uint32_t* d_posmask = nullptr; // [dim/2] bf16x2 sign-bit masks indexed by ROTATED position: bit 15 / bit 31 set where
+                                 // position 2i / 2i+1 has sign -1
 };
 
 namespace oq {
@@ -63,6 +65,10 @@ int* device_status_word();   // device pointer (allocated on first use), or null
 int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_codebook* cb_a,
                    const void* Wq_idx, const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y,
                    int ldy, int y_dtype, int* status, void* stream);
+// Rotate+quantize of activations with an explicit status word (NULL: the library's own, allocated on first use).
+int rotate_quantize_act_launch(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                               const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated, int* status,
+                               void* stream);
 // Status word of the allocation-free entry point on the current device, or nullptr before its first call.
 int* noalloc_status_word();
 

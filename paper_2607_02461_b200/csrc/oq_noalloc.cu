@@ -73,7 +73,7 @@ extern "C" int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int d
   // The rotation's device tables are uploaded (and allocated) by the first ordinary GPU call that uses the
   // handle -- in practice oq_quantize_weights, which has to run before any forward pass.  This entry point
   // must not allocate, so it refuses a handle that has never been on the device.
-  if (!rot->d_offset || !rot->d_gather || !rot->d_srcmask)
+  if (!rot->d_offset || !rot->d_gather || !rot->d_srcmask || !rot->d_posmask)
     return fail(OQ_ERR_INVALID_ARG,
                 "oq_linear_forward_noalloc: the rotation handle has no device tables yet (they are created by the first "
                 "oq_quantize_weights / oq_rotate_quantize_act call with this handle)");
@@ -83,7 +83,7 @@ extern "C" int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int d
   int* status = reinterpret_cast<int*>(scratch);
   float* norms = reinterpret_cast<float*>(scratch + kNormOffset);
   void* idx = scratch + kIdxOffset;
-  rc = oq_rotate_quantize_act(X_bf16, n_tokens, dim, ldx, rot, cb_a, idx, norms, nullptr, stream);
+  rc = rotate_quantize_act_launch(X_bf16, n_tokens, dim, ldx, rot, cb_a, idx, norms, nullptr, status, stream);
   if (rc != OQ_OK) return rc;
   return qlinear_launch(idx, norms, n_tokens, cb_a, Wq_idx, Wq_norm_bf16, m, cb_w, dim, Y, ldy, y_dtype, status, stream);
 }

@@ -5,6 +5,7 @@
 #include "oq_internal.h"
 #include "oq_packing.cuh"
 #include "oq_rq_fast.cuh"
+#include "oq_rq_tc.cuh"
 
 namespace oq {
 
@@ -183,9 +184,59 @@ static cudaError_t launch_fast_T(int bits, int grid, const FastPlan& pl, cudaStr
   return cudaErrorInvalidValue;
 }
 
+// Which rotate+quantize kernel to use: 0 = choose by shape, 1 = general, 2 = register butterflies, 3 = tensor
+// cores.  A forced kernel that cannot handle the shape falls back to the general one.
+static int g_forced_kernel = 0;
+
+// Plan of the tensor-core kernel: rows per group T (a power of two <= 16) such that the T * dim / 128 (token,
+// block) pairs of a group fill as much as possible of at most four 128-row tiles and the rows fit in shared
+// memory beside the Hadamard tile and two operand tiles.
+struct TcPlan {
+  int tshift, ntiles, tmem_cols;
+  bool tab_smem;
+  size_t smem;
+  double fill;
+};
+static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
+  if (block != 128 || !cb->poly.ok) return false;
+  const size_t kMaxSmem = 227 * 1024;
+  const int kblocks = dim / 128;
+  bool found = false;
+  for (int ts = 4; ts >= 0; --ts) {
+    const int T = 1 << ts;
+    const int pairs = T * kblocks;
+    const int ntiles = (pairs + 127) / 128;
+    if (ntiles > 4) continue;
+    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)T * rqtc::row_pitch_bytes(dim) + 16 * 16 * 4 + 128;
+    const size_t with_tab = base + 6 * (size_t)dim;
+    if (base > kMaxSmem) continue;
+    const double fill = (double)pairs / (128.0 * ntiles);
+    if (found && fill <= plan->fill + 1e-9) continue;
+    plan->tshift = ts;
+    plan->ntiles = ntiles;
+    plan->tmem_cols = ntiles == 1 ? 128 : ntiles == 2 ? 256 : 512;
+    plan->tab_smem = with_tab <= kMaxSmem;
+    plan->smem = plan->tab_smem ? with_tab : base;
+    // never two of these CTAs on one SM: they would wait for each other's tensor memory
+    if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
+    plan->fill = fill;
+    found = true;
+  }
+  return found;
+}
+
+template <int BITS>
+static cudaError_t launch_tc_bits(bool tab_smem, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
+  auto k = tab_smem ? rq_tc_kernel<BITS, true> : rq_tc_kernel<BITS, false>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  k<<<grid, rqtc::THREADS, smem, st>>>(prm);
+  return cudaGetLastError();
+}
+
 template <bool kBf16Norm>
 static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, const oq_rpbh* rot,
-                     const oq_codebook* cb, void* out_idx, void* out_norm, float* dbg, void* stream) {
+                     const oq_codebook* cb, void* out_idx, void* out_norm, float* dbg, int* status, void* stream) {
   int rc = check_common(fn, X, rows, dim, ld, rot, cb, out_idx, out_norm);
   if (rc != OQ_OK || rows == 0) return rc;
   rc = ensure_device_tables(rot);
@@ -197,8 +248,31 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
   cudaGetDevice(&dev);
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  TcPlan tp;
+  const bool tc_ok = plan_tc(dim, rot->block, cb, &tp);
+  if ((g_forced_kernel == 0 && tc_ok && tp.fill >= 0.6) || (g_forced_kernel == 3 && tc_ok)) {
+    if (!status) status = device_status_word();
+    if (!status) return fail(OQ_ERR_CUDA, std::string(fn) + ": cannot allocate the device status word");
+    RqTcParams prm;
+    prm.X = reinterpret_cast<const unsigned char*>(X);
+    prm.rows = rows; prm.dim = dim; prm.ldx = ld;
+    prm.offset = rot->d_offset; prm.posmask = rot->d_posmask;
+    prm.out_idx = reinterpret_cast<uint32_t*>(out_idx); prm.pitch_words = pitch_words;
+    prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
+    const int T = 1 << tp.tshift;
+    prm.groups = (rows + T - 1) / T;
+    prm.tshift = tp.tshift; prm.ntiles = tp.ntiles; prm.tmem_cols = tp.tmem_cols;
+    prm.bf16_norm = kBf16Norm ? 1 : 0;
+    prm.status = status;
+    int grid = sms < prm.groups ? sms : prm.groups;
+    if (cb->bits == 4) e = launch_tc_bits<4>(tp.tab_smem, grid, tp.smem, st, prm);
+    else if (cb->bits == 3) e = launch_tc_bits<3>(tp.tab_smem, grid, tp.smem, st, prm);
+    else e = launch_tc_bits<2>(tp.tab_smem, grid, tp.smem, st, prm);
+    if (e != cudaSuccess) return cuda_fail(e, fn);
+    return OQ_OK;
+  }
   FastPlan pl;
-  if (plan_fast(dim, rot->block, cb, &pl)) {
+  if (g_forced_kernel != 1 && plan_fast(dim, rot->block, cb, &pl)) {
     RqFastParams prm;
     prm.X = reinterpret_cast<const uint32_t*>(X);
     prm.rows = rows; prm.dim = dim; prm.ldw = ld / 2;
@@ -234,6 +308,13 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
   return OQ_OK;
 }
 
+int rotate_quantize_act_launch(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                               const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated, int* status,
+                               void* stream) {
+  return launch_rq<false>("oq_rotate_quantize_act", X_bf16, n_tokens, dim, ldx, rot, cb_a, Xq_idx, Xq_norm,
+                          dbg_rotated, status, stream);
+}
+
 }  // namespace oq
 
 using namespace oq;
@@ -243,14 +324,20 @@ extern "C" {
 int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
                            const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated,
                            void* stream) {
-  return launch_rq<false>("oq_rotate_quantize_act", X_bf16, n_tokens, dim, ldx, rot, cb_a, Xq_idx, Xq_norm,
-                          dbg_rotated, stream);
+  return rotate_quantize_act_launch(X_bf16, n_tokens, dim, ldx, rot, cb_a, Xq_idx, Xq_norm, dbg_rotated, nullptr,
+                                    stream);
+}
+
+int oq_debug_select_rq_kernel(int which) {
+  if (which < 0 || which > 3) return fail(OQ_ERR_INVALID_ARG, "oq_debug_select_rq_kernel: which must be 0..3");
+  g_forced_kernel = which;
+  return OQ_OK;
 }
 
 int oq_quantize_weights(const void* W_bf16, int m, int dim, int ldw, const oq_rpbh* rot, const oq_codebook* cb_w,
                         void* Wq_idx, void* Wq_norm_bf16, void* dbg_rotated, void* stream) {
   return launch_rq<true>("oq_quantize_weights", W_bf16, m, dim, ldw, rot, cb_w, Wq_idx, Wq_norm_bf16,
-                         reinterpret_cast<float*>(dbg_rotated), stream);
+                         reinterpret_cast<float*>(dbg_rotated), nullptr, stream);
 }
 
 int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream) {

@@ -79,8 +79,10 @@ def main(argv=None):
     ap.add_argument("--block", type=int, default=128)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--kernel", type=int, default=0, help="rotate+quantize kernel: 0 auto, 1 general, 2 registers, 3 tensor cores")
     a = ap.parse_args(argv)
     oqbuild.build()
+    B.oq_debug_select_rq_kernel(a.kernel)
     if a.mode == "rq":
         print(json.dumps(run_rq(a.tokens, a.dim, a.bits, a.block, a.iters)))
     elif a.mode == "gemm":

@@ -20,7 +20,16 @@ def _dev(bits_u16):
     return torch.from_numpy(bits_u16.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def check_rows(xb, block, seed, bits, weights=False, rows=None):
+AUTO, GENERAL, REGISTERS, TENSOR = 0, 1, 2, 3    # oq_debug_select_rq_kernel
+
+
+@pytest.fixture(autouse=True)
+def _default_kernel_afterwards():
+    yield
+    B.oq_debug_select_rq_kernel(AUTO)
+
+
+def check_rows(xb, block, seed, bits, weights=False, rows=None, kernel=AUTO):
     """Runs the GPU pass on xb (uint16 bf16 bits [N, d]) and compares with the oracle on `rows`."""
     import torch
     n, d = xb.shape
@@ -28,7 +37,9 @@ def check_rows(xb, block, seed, bits, weights=False, rows=None):
     X = _dev(xb)
     dbg = torch.full((n, d), float("nan"), dtype=torch.float32, device="cuda")
     fn = B.oq_quantize_weights if weights else B.oq_rotate_quantize_act
+    B.oq_debug_select_rq_kernel(kernel)
     idx_p, norm = fn(X, rot, cb, dbg_rotated=dbg)
+    B.oq_debug_select_rq_kernel(AUTO)
     idx = B.oq_unpack_indices(idx_p, n, d, bits).cpu().numpy()
     torch.cuda.synchronize()
     assert B.oq_device_status() == 0
@@ -70,6 +81,38 @@ def test_activation_rows_match_oracle(d, block, bits):
     xb = synth.activations(67 if d < 8000 else 21, d, seed=1000 + bits)   # ragged against any row tiling
     rate = check_rows(xb, block, 0, bits)
     assert rate <= 1e-4
+
+
+@pytest.mark.parametrize("kernel", [GENERAL, REGISTERS, TENSOR])
+@pytest.mark.parametrize("bits", [4, 3, 2])
+@pytest.mark.parametrize("d,n", [(128, 67), (256, 40), (1024, 67), (3072, 67), (5120, 35), (12288, 21), (13824, 9)])
+def test_every_kernel_matches_oracle_on_blocks_of_128(d, n, bits, kernel):
+    """The three kernels compute the same function; blocks of 128 are the shape all of them support."""
+    xb = synth.activations(n, d, seed=1100 + bits)
+    assert check_rows(xb, 128, 1, bits, kernel=kernel) <= 1e-4
+
+
+@pytest.mark.parametrize("kernel", [REGISTERS, TENSOR])
+def test_kernels_agree_with_each_other_on_many_groups(kernel):
+    """More row groups than CTAs (several pipeline rounds per CTA), ragged last group: same packed words and
+    norms (to rounding) as the general kernel."""
+    import torch
+    d, n = 1024, 148 * 16 * 3 + 5
+    xb = synth.activations(n, d, seed=1200)
+    rot, cb = B.oq_make_rpbh(d, 128, 2), B.oq_build_codebook(d, 4)
+    X = _dev(xb)
+    B.oq_debug_select_rq_kernel(GENERAL)
+    ref_idx, ref_norm = B.oq_rotate_quantize_act(X, rot, cb)
+    B.oq_debug_select_rq_kernel(kernel)
+    idx, norm = B.oq_rotate_quantize_act(X, rot, cb)
+    B.oq_debug_select_rq_kernel(AUTO)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.allclose(norm, ref_norm, rtol=2e-6, atol=0)
+    a = B.oq_unpack_indices(idx, n, d, 4).to(torch.int16)
+    b = B.oq_unpack_indices(ref_idx, n, d, 4).to(torch.int16)
+    diff = (a - b).abs()
+    assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 1e-4
 
 
 def test_config1_single_linear_activation_side():
@@ -122,11 +165,13 @@ def test_empty_and_bad_arguments():
     assert e.value.code == 3
 
 
-def test_results_are_deterministic():
+@pytest.mark.parametrize("kernel", [AUTO, REGISTERS, TENSOR])
+def test_results_are_deterministic(kernel):
     import torch
     xb = synth.activations(300, 3072, seed=1001)
     rot, cb = B.oq_make_rpbh(3072, 128, 0), B.oq_build_codebook(3072, 4)
     X = _dev(xb)
+    B.oq_debug_select_rq_kernel(kernel)
     a = B.oq_rotate_quantize_act(X, rot, cb)
     b = B.oq_rotate_quantize_act(X, rot, cb)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
