@@ -207,8 +207,8 @@ static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
     const int pairs = T * kblocks;
     const int ntiles = (pairs + 127) / 128;
     if (ntiles > 4) continue;
-    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)T * rqtc::row_pitch_bytes(dim) + 16 * 16 * 4 + 128;
-    const size_t with_tab = base + 6 * (size_t)dim;
+    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)T * rqtc::row_pitch_bytes(dim) + 16 * 16 * 4 + 128;   // + partial sums, barriers, counters
+    const size_t with_tab = base + (size_t)kblocks * 4 * (rqtc::TAB_PITCH + rqtc::MSK_PITCH);
     if (base > kMaxSmem) continue;
     const double fill = (double)pairs / (128.0 * ntiles);
     if (found && fill <= plan->fill + 1e-9) continue;

@@ -144,28 +144,33 @@ __device__ __forceinline__ void sign_sources(const float* z, uint32_t* s) {
 
 __device__ __forceinline__ uint32_t sign_source(float z) { return __float_as_uint(z - __uint_as_float(1u)); }
 
+// One word of the 4-bit format: 8 consecutive rotated coordinates.  Nibbles are emitted from 7 down to 0; nibble n
+// carries the magnitude of coordinate n and, in its top bit, the sign of coordinate (n odd ? (n-1)/2 : 4 + n/2).
+__device__ __forceinline__ uint32_t pack8_4bit(const float* z, float kappa, const Poly2<7>& poly) {
+  constexpr uint32_t MAGIC = 0x4B400000u;
+  uint32_t sgn[8], lvl[8];
+  sign_sources<8>(z, sgn);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) poly.eval(z[2 * i], z[2 * i + 1], kappa, lvl[2 * i], lvl[2 * i + 1]);
+  uint32_t word = 0;
+#pragma unroll
+  for (int n = 7; n >= 0; --n) {
+    const int se = (n & 1) ? (n - 1) / 2 : 4 + n / 2;            // whose sign rides in nibble n
+    word = __funnelshift_l(sgn[se], word, 1);
+    word = (word << 3) + lvl[n];
+  }
+  // every step added MAGIC at nibble position n: remove MAGIC * (16^0 + ... + 16^7) (mod 2^32)
+  return word - MAGIC * 0x11111111u;
+}
+
 // Packs 32 consecutive rotated coordinates z[0..32) of one row into BITS words.
 template <int BITS>
 __device__ __forceinline__ void pack32(const float* z, float kappa, const Poly2<(1 << (BITS - 1)) - 1>& poly,
                                        uint32_t* out) {
-  constexpr uint32_t MAGIC = 0x4B400000u;
-  if (BITS == 4) {
+  [[maybe_unused]] constexpr uint32_t MAGIC = 0x4B400000u;
+  if constexpr (BITS == 4) {
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      uint32_t sgn[8], lvl[8];
-      sign_sources<8>(z + 8 * w, sgn);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) poly.eval(z[8 * w + 2 * i], z[8 * w + 2 * i + 1], kappa, lvl[2 * i], lvl[2 * i + 1]);
-      uint32_t word = 0;
-#pragma unroll
-      for (int n = 7; n >= 0; --n) {
-        const int se = (n & 1) ? (n - 1) / 2 : 4 + n / 2;            // whose sign rides in nibble n
-        word = __funnelshift_l(sgn[se], word, 1);
-        word = (word << 3) + lvl[n];
-      }
-      // every step added MAGIC at nibble position n: remove MAGIC * (16^0 + ... + 16^7) (mod 2^32)
-      out[w] = word - MAGIC * 0x11111111u;
-    }
+    for (int w = 0; w < 4; ++w) out[w] = pack8_4bit(z + 8 * w, kappa, poly);
   } else {
     // sign word: coordinate k' sits at bit 8(k'&3) + 7 - (k'>>2); emit bits 31 .. 0
     uint32_t sw = 0;
