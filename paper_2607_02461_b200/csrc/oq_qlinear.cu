@@ -269,7 +269,9 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
                     CodebookParams cba, CodebookParams cbw, void* __restrict__ Y, int ldy, int* status) {
   using namespace pair;
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  // 1024-byte alignment computed on the shared-window address: the compiler keeps treating the tiles as shared
+  // memory (32-bit addresses) instead of falling back to generic-pointer arithmetic
+  unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + PSTAGES * PSTAGE_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PSTAGES + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
