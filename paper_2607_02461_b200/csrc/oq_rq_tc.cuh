@@ -9,8 +9,8 @@
 // norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.
 //
 // Data flow per CTA (persistent over groups of T consecutive rows, T a power of two <= 16):
-//   copy      a bulk copy per row (global -> shared, 16-byte aligned row pitch) and an L2 prefetch for the group
-//             after; the rows of the next group are requested by whichever warp is the last to finish the
+//   copy      a bulk copy per row (global -> shared, 16-byte aligned row pitch); the rows of the next group are
+//             requested by whichever warp is the last to finish the
 //             shared-memory loads of this group's last tile;
 //   gather    512 threads; a thread owns one of the 128 (token, block) pairs of a tile and 32 of its rotated
 //             coordinates: table look-up, 16-bit shared-memory load, pair-wise sign mask, 16-byte store into
@@ -90,6 +90,21 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rows_full = smem_u32(bars), acc_ready0 = smem_u32(bars + 1);
 
+  const int kblocks = p.dim / H;
+  const uint32_t row_bytes = 2u * (uint32_t)p.dim;
+  const int stride = (int)gridDim.x;
+  // Bulk copies of the rows of group `grp` into the row buffer.
+  auto request_rows = [&](int grp) {
+    const int row0 = grp * T;
+    const int nvalid = min(T, p.rows - row0);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(rows_full), "r"(row_bytes * (uint32_t)nvalid) : "memory");
+    for (int r = 0; r < nvalid; ++r) {
+      const unsigned char* src = p.X + (size_t)(row0 + r) * p.ldx * 2;
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(rows_s + (size_t)r * pitch)), "l"(src), "r"(row_bytes), "r"(rows_full) : "memory");
+    }
+    s_cnt[3] += 1u;
+  };
   if (tid == 0) {
     mbar_init(rows_full, 1);
     for (int i = 0; i < 4; ++i) mbar_init(acc_ready0 + 8 * i, 1);                   // tcgen05.commit
@@ -97,6 +112,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     for (int i = 0; i < 4; ++i) s_cnt[i] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // the first rows travel while the CTA builds its tables
+    if ((int)blockIdx.x < p.groups) request_rows(blockIdx.x);
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
@@ -125,32 +142,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
-  const int kblocks = p.dim / H;
-  const uint32_t row_bytes = 2u * (uint32_t)p.dim;
-  const int stride = (int)gridDim.x;
 
-  // Bulk copies of the rows of group `grp` into the row buffer, and an L2 prefetch of the group after it.
-  auto request_rows = [&](int grp) {
-    const int row0 = grp * T;
-    const int nvalid = min(T, p.rows - row0);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(rows_full), "r"(row_bytes * (uint32_t)nvalid) : "memory");
-    for (int r = 0; r < nvalid; ++r) {
-      const unsigned char* src = p.X + (size_t)(row0 + r) * p.ldx * 2;
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(rows_s + (size_t)r * pitch)), "l"(src), "r"(row_bytes), "r"(rows_full) : "memory");
-    }
-    s_cnt[3] += 1u;
-    const int after = grp + stride;
-    if (after < p.groups) {
-      const int arow0 = after * T;
-      const int an = min(T, p.rows - arow0);
-      for (int r = 0; r < an; ++r) {
-        const unsigned char* src = p.X + (size_t)(arow0 + r) * p.ldx * 2;
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(row_bytes) : "memory");
-      }
-    }
-  };
-  if (tid == 0 && (int)blockIdx.x < p.groups) request_rows(blockIdx.x);
 
   const int q = warp & 3, kq = warp >> 2;          // tensor-memory lane quarter, column quarter
   const int r = q * 32 + lane;                     // row of the operand tile = tensor-memory lane
