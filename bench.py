@@ -334,7 +334,7 @@ def run_ours(args):
                      "frac_of_nominal_2250": gemm_tf / 2250.0,
                      "per_layer_tflops": {l["name"]: 2 * tokens * l["m"] * l["d"] / (gemm_ms[i] * 1e-3) / 1e12
                                           for i, l in enumerate(L)}},
-        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq_fast_kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
+        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq_tc_kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
                                      "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
                                      "traffic": (traffic or {}).get("rq_bytes_per_step"),
                                      "algorithmic_bytes_per_step": rq_b, "frac_of_nominal_8000": rq_gbs / 8000.0,
