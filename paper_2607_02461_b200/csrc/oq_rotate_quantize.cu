@@ -188,46 +188,44 @@ static cudaError_t launch_fast_T(int bits, int grid, const FastPlan& pl, cudaStr
 // cores.  A forced kernel that cannot handle the shape falls back to the general one.
 static int g_forced_kernel = 0;
 
-// Plan of the tensor-core kernel: rows per group T (a power of two <= 16) such that the T * dim / 128 (token,
-// block) pairs of a group fill as much as possible of at most four 128-row tiles and the rows fit in shared
-// memory beside the Hadamard tile and two operand tiles.
+// Plan of the tensor-core kernel: th tokens per half group (1, 2, 4 or 8), the largest for which the
+// P = th * dim / 128 (token, block) pairs of a half number at most 192 and three half groups of rows fit in
+// shared memory beside the Hadamard tile.
 struct TcPlan {
-  int tshift, ntiles, tmem_cols;
-  bool tab_smem;
+  int ths, pairs, ntiles;
+  int tab;          // 0: tables in global memory, 1: both in shared memory, 2: 16-bit offsets in shared memory
   size_t smem;
-  double fill;
+  double fill;      // used rows of the operand tiles / all rows
 };
 static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
   if (block != 128 || !cb->poly.ok) return false;
   const size_t kMaxSmem = 227 * 1024;
   const int kblocks = dim / 128;
-  bool found = false;
-  for (int ts = 4; ts >= 0; --ts) {
-    const int T = 1 << ts;
-    const int pairs = T * kblocks;
-    const int ntiles = (pairs + 127) / 128;
-    if (ntiles > 4) continue;
-    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)T * rqtc::row_pitch_bytes(dim) + 16 * 16 * 4 + 128;   // + partial sums, barriers, counters
-    const size_t with_tab = base + (size_t)kblocks * 4 * (rqtc::TAB_PITCH + rqtc::MSK_PITCH);
+  for (int ths = 3; ths >= 0; --ths) {
+    const int th = 1 << ths;
+    const int pairs = th * kblocks;
+    if (pairs > rqtc::MAX_PAIRS) continue;
+    // + partial sums, barriers, counters
+    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)rqtc::ROWBUFS * th * rqtc::row_pitch_bytes(dim) + 2 * 16 * 16 * 4 + 256;
     if (base > kMaxSmem) continue;
-    const double fill = (double)pairs / (128.0 * ntiles);
-    if (found && fill <= plan->fill + 1e-9) continue;
-    plan->tshift = ts;
-    plan->ntiles = ntiles;
-    plan->tmem_cols = ntiles == 1 ? 128 : ntiles == 2 ? 256 : 512;
-    plan->tab_smem = with_tab <= kMaxSmem;
-    plan->smem = plan->tab_smem ? with_tab : base;
+    const size_t with_tab = base + (size_t)kblocks * 4 * (rqtc::TAB_PITCH + rqtc::MSK_PITCH);
+    const size_t with_tab16 = base + (size_t)kblocks * 4 * rqtc::MSK_PITCH;   // byte offsets fit 16 bits: dim < 32768
+    plan->ths = ths;
+    plan->pairs = pairs;
+    plan->ntiles = pairs <= 128 ? 2 : 3;
+    plan->tab = with_tab <= kMaxSmem ? 1 : (with_tab16 <= kMaxSmem && dim < 32768) ? 2 : 0;
+    plan->smem = plan->tab == 1 ? with_tab : plan->tab == 2 ? with_tab16 : base;
     // never two of these CTAs on one SM: they would wait for each other's tensor memory
     if (plan->smem < 120 * 1024) plan->smem = 120 * 1024;
-    plan->fill = fill;
-    found = true;
+    plan->fill = 2.0 * pairs / (128.0 * plan->ntiles);
+    return true;
   }
-  return found;
+  return false;
 }
 
 template <int BITS>
-static cudaError_t launch_tc_bits(bool tab_smem, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
-  auto k = tab_smem ? rq_tc_kernel<BITS, true> : rq_tc_kernel<BITS, false>;
+static cudaError_t launch_tc_bits(int tab, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
+  auto k = tab == 1 ? rq_tc_kernel<BITS, 1> : tab == 2 ? rq_tc_kernel<BITS, 2> : rq_tc_kernel<BITS, 0>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   k<<<grid, rqtc::THREADS, smem, st>>>(prm);
@@ -259,15 +257,15 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
     prm.offset = rot->d_offset; prm.posmask = rot->d_posmask;
     prm.out_idx = reinterpret_cast<uint32_t*>(out_idx); prm.pitch_words = pitch_words;
     prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
-    const int T = 1 << tp.tshift;
+    const int T = 2 << tp.ths;
     prm.groups = (rows + T - 1) / T;
-    prm.tshift = tp.tshift; prm.ntiles = tp.ntiles; prm.tmem_cols = tp.tmem_cols;
+    prm.ths = tp.ths; prm.pairs = tp.pairs; prm.ntiles = tp.ntiles;
     prm.bf16_norm = kBf16Norm ? 1 : 0;
     prm.status = status;
     int grid = sms < prm.groups ? sms : prm.groups;
-    if (cb->bits == 4) e = launch_tc_bits<4>(tp.tab_smem, grid, tp.smem, st, prm);
-    else if (cb->bits == 3) e = launch_tc_bits<3>(tp.tab_smem, grid, tp.smem, st, prm);
-    else e = launch_tc_bits<2>(tp.tab_smem, grid, tp.smem, st, prm);
+    if (cb->bits == 4) e = launch_tc_bits<4>(tp.tab, grid, tp.smem, st, prm);
+    else if (cb->bits == 3) e = launch_tc_bits<3>(tp.tab, grid, tp.smem, st, prm);
+    else e = launch_tc_bits<2>(tp.tab, grid, tp.smem, st, prm);
     if (e != cudaSuccess) return cuda_fail(e, fn);
     return OQ_OK;
   }

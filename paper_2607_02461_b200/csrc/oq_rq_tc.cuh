@@ -8,22 +8,30 @@
 // accumulated in fp32 in tensor memory).  The rest of the path reads tensor memory twice: once for the row
 // norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.
 //
-// Data flow per CTA (persistent over groups of T consecutive rows, T a power of two <= 16):
-//   copy      a bulk copy per row (global -> shared, 16-byte aligned row pitch); the rows of the next group are
-//             requested by whichever warp is the last to finish the
-//             shared-memory loads of this group's last tile;
-//   gather    512 threads; a thread owns one of the 128 (token, block) pairs of a tile and 32 of its rotated
-//             coordinates: table look-up, 16-bit shared-memory load, pair-wise sign mask, 16-byte store into
-//             the K-major 128-byte-swizzled operand tile (two tile buffers);
-//   mma       the warp that finishes a tile last issues 8 x tcgen05.mma (M = 128 pairs, N = 128 coordinates,
-//             K = 16) into the tile's own 128-column accumulator (a group's whole rotated output stays in
-//             tensor memory) and commits to a barrier;
-//   pass 1    every thread reads its 32 columns of every tile, sums squares; partial sums meet in shared
-//             memory in a fixed order (deterministic norms);
-//   pass 2    reads the same columns again, finds the levels with the polynomial of QuantPoly, packs, stores.
-//             It is fused with the gather of the NEXT group, 8 coordinates at a time: the level search keeps
-//             the FMA and ALU pipes busy while the gather waits for shared memory.
-// Every wait is bounded and reports to a status word.
+// Work units.  A group is 2 th consecutive rows (th = 1, 2, 4 or 8 tokens per HALF group, chosen so that the
+// P = th * dim / 128 (token, block) pairs of a half number at most 192).  Each half has its own row buffer and
+// its own "rows landed" barrier.  The pairs of a group fill two or three operand tiles of 128 rows:
+//     P <= 128:  tile 0 = half 0,  tile 1 = half 1;
+//     P >  128:  tile 0 = first 128 pairs of half 0,  tile 2 = first 128 pairs of half 1,
+//                tile 1 = the remaining pairs of half 0 (rows 0..63) and of half 1 (rows 64..127).
+// Tiles are gathered in the order 0, 1, 2, so half 0's buffer is free one tile before half 1's and the copy of
+// each half of the next group overlaps the gather of the other half.
+//
+// Warp roles (25 warps, every wait bounded, reporting to a status word):
+//   gather  (8 warps)  a thread owns one row of a tile (a pair) and 64 of its rotated coordinates: offset table,
+//                      16-bit shared-memory load (the th tokens of a warp sit in different banks), pair-wise sign
+//                      mask, 16-byte stores into the K-major 128-byte-swizzled operand tile (two tile buffers).
+//                      The warp that is the last to finish a half's loads requests the bulk copies (one per row,
+//                      16-byte aligned pitch) of that half of the CTA's next group.  These warps run ahead of
+//                      the others by up to two operand tiles / four accumulators;
+//   mma     (1 thread) per tile: 8 x tcgen05.mma (M = 128 pairs, N = 128 coordinates, K = 16) into one of four
+//                      128-column accumulators in tensor memory, committed to "accumulator ready" and
+//                      "tile buffer free";
+//   compute (16 warps) pass 1: every thread reads its 32 columns of every tile of a group and sums squares;
+//                      partial sums meet in shared memory in a fixed order (deterministic norms);
+//                      pass 2: reads the same columns again, finds the levels with the polynomial of QuantPoly,
+//                      packs, stores, and frees the accumulator.
+// Gather warps wait on shared memory, compute warps on the FMA and ALU pipes: the warp schedulers overlap them.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -43,80 +51,109 @@ struct RqTcParams {
   void* out_norm;
   float* dbg;
   QuantPoly poly;
-  int groups;               // number of T-row groups
-  int tshift;               // log2(T)
-  int ntiles;               // tiles of 128 (token, block) pairs per group (1..4)
-  int tmem_cols;            // 128 * ntiles rounded up to a power of two
+  int groups;               // number of groups of 2 th rows
+  int ths;                  // log2(th), th = tokens per half group
+  int pairs;                // P = th * dim / 128 pairs per half (<= 192)
+  int ntiles;               // 2 (P <= 128) or 3
   int bf16_norm;            // 1: norms stored as bf16 (weights), 0: fp32 (activations)
   int* status;
 };
 
 namespace rqtc {
 constexpr int H = 128;
-constexpr int THREADS = 512;                      // 16 warps: 4 lane quarters x 4 column quarters of a tile
-constexpr int WARPS = THREADS / 32;
+constexpr int COMPUTE_WARPS = 16;                 // 4 lane quarters x 4 column quarters of a tile
+constexpr int GATHER_WARPS = 8;                   // 4 lane quarters x 2 halves of the 128 coordinates
+constexpr int COMPUTE_THREADS = COMPUTE_WARPS * 32;
+constexpr int THREADS = (COMPUTE_WARPS + GATHER_WARPS + 1) * 32;
+constexpr int MMA_WARP = COMPUTE_WARPS + GATHER_WARPS;
+constexpr int SLOTS = 3;                          // accumulators of 128 columns in tensor memory
+constexpr int ABUFS = 2;                          // operand tiles in tensor memory: 128 lanes x 64 columns of bf16 pairs
+constexpr uint32_t A_COL0 = SLOTS * 128;          // first column of the operand tiles
+constexpr int TMEM_COLS = 512;
+constexpr int ROWBUFS = 3;                        // row buffers, one half group each
 constexpr uint32_t ATOM = 128 * 128;              // 128 rows x 64 bf16: one swizzle atom column of a tile
 constexpr uint32_t TILE = 2 * ATOM;               // 128 rows x 128 bf16
-constexpr uint32_t OFF_H = 0, OFF_A = TILE, OFF_ROWS = 3 * TILE;
+constexpr uint32_t OFF_H = 0, OFF_ROWS = TILE;
 constexpr int TAB_PITCH = 132, MSK_PITCH = 68;    // words per block of the shared-memory table copies
-enum { WAIT_ROWS = 11, WAIT_ACC = 13, WAIT_DRAIN = 14 };
+constexpr int MAX_PAIRS = 192;
+enum { WAIT_ROWS = 11, WAIT_AFULL = 12, WAIT_ACC = 13, WAIT_DRAIN = 14, WAIT_AFREE = 15, WAIT_ACCFREE = 16 };
 __host__ __device__ constexpr uint32_t row_pitch_bytes(int dim) { return 2u * (uint32_t)dim + 16u; }
 }  // namespace rqtc
 
-
-template <int BITS, bool TAB_SMEM>
+// TAB: where the gather tables live.  0: global memory (read-only path); 1: both copied to shared memory (32-bit
+// offsets, masks); 2: offsets copied to shared memory as 16-bit values, masks stay in global memory.
+template <int BITS, int TAB>
 __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParams p) {
   using namespace rqtc;
   extern __shared__ unsigned char smem_dyn[];
   // 1024-byte alignment for the swizzled tiles, computed on the shared-window address so that the compiler keeps
   // treating everything below as shared memory (32-bit addresses, no generic-pointer arithmetic)
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-  const int T = 1 << p.tshift;
+  const int th = 1 << p.ths, T = 2 * th;
   const uint32_t pitch = row_pitch_bytes(p.dim);
-  unsigned char* rows_s = smem + OFF_ROWS;
-  unsigned char* after_rows = rows_s + (size_t)T * pitch;
-  // copies of the offset and sign-mask tables (TAB_SMEM): the 128 / 64 words of a block are followed by 4 words
-  // of padding, so that the four blocks a warp reads at once sit in different banks
-  uint32_t* s_table = reinterpret_cast<uint32_t*>(after_rows);                                 // [dim/128][TAB_PITCH]
-  uint32_t* s_mask = s_table + (TAB_SMEM ? (p.dim / H) * TAB_PITCH : 0);                       // [dim/128][MSK_PITCH]
-  float* s_part = reinterpret_cast<float*>(s_mask + (TAB_SMEM ? (p.dim / H) * MSK_PITCH : 0)); // [16 warps][16]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_part + WARPS * 16);                           // rows_full, acc_ready[4]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+  unsigned char* rows_s = smem + OFF_ROWS;          // [3 buffers][th rows][pitch]
+  unsigned char* after_rows = rows_s + (size_t)ROWBUFS * th * pitch;
+  // copies of the offset and sign-mask tables: the words of a block are followed by 4 words of padding, so that
+  // the blocks a warp reads at once sit in different banks
+  uint32_t* s_table = reinterpret_cast<uint32_t*>(after_rows);    // [dim/128][TAB_PITCH] (TAB 1) or [dim/128][MSK_PITCH] (TAB 2)
+  uint32_t* s_mask = s_table + (TAB == 1 ? (p.dim / H) * TAB_PITCH : TAB == 2 ? (p.dim / H) * MSK_PITCH : 0);   // [dim/128][MSK_PITCH] (TAB 1)
+  float* s_part = reinterpret_cast<float*>(s_mask + (TAB == 1 ? (p.dim / H) * MSK_PITCH : 0));                  // [2][16 warps][2 halves][8]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_part + 2 * COMPUTE_WARPS * 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  // arrival counters (never reset; the warp that brings one to a multiple of 16 acts): [0], [1] operand tile
-  // buffers finished, [2] row buffer no longer needed, [3] row groups requested so far
+  // [0..2]: gather warps that no longer need row buffer b (never reset; the warp that brings one to a multiple of
+  // 8 requests the next copy into it); [3..5]: copies requested per buffer
   unsigned int* s_cnt = reinterpret_cast<unsigned int*>(tmem_slot + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t rows_full = smem_u32(bars), acc_ready0 = smem_u32(bars + 1);
-
-  const int kblocks = p.dim / H;
+  const uint32_t rows_full0 = smem_u32(bars);          // [3] bulk copies of a half group have landed in buffer b
+  const uint32_t a_full0 = smem_u32(bars + 3);         // [2] operand tile written by the 8 gather warps
+  const uint32_t a_free0 = smem_u32(bars + 5);         // [2] operand tile read by its MMAs
+  const uint32_t acc_ready0 = smem_u32(bars + 7);      // [3] accumulator written by its MMAs
+  const uint32_t acc_free0 = smem_u32(bars + 10);      // [3] accumulator read twice by the 16 compute warps
   const uint32_t row_bytes = 2u * (uint32_t)p.dim;
   const int stride = (int)gridDim.x;
-  // Bulk copies of the rows of group `grp` into the row buffer.
-  auto request_rows = [&](int grp) {
-    const int row0 = grp * T;
-    const int nvalid = min(T, p.rows - row0);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(rows_full), "r"(row_bytes * (uint32_t)nvalid) : "memory");
+  const bool nt3 = p.ntiles == 3;
+  const int rem = p.pairs - 128;     // pairs of a half that go to the shared middle tile (nt3)
+
+  // Half groups are numbered hs = 2 * (index of the group within this CTA) + half and live in row buffer hs % 3.
+  // Bulk copies of half group hs into its buffer; one that lies past the last row (or past the last group) still
+  // completes its barrier phase (0 bytes).
+  auto request_half = [&](uint32_t hs) {
+    const uint32_t b = hs % 3u;
+    const uint32_t bar = rows_full0 + 8 * b;
+    const long long grp = (long long)blockIdx.x + (long long)(hs >> 1) * stride;
+    const long long row0 = grp * T + (long long)(hs & 1u) * th;
+    const int nvalid = grp < p.groups ? (int)max(0ll, min((long long)th, (long long)p.rows - row0)) : 0;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(row_bytes * (uint32_t)nvalid) : "memory");
     for (int r = 0; r < nvalid; ++r) {
       const unsigned char* src = p.X + (size_t)(row0 + r) * p.ldx * 2;
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(rows_s + (size_t)r * pitch)), "l"(src), "r"(row_bytes), "r"(rows_full) : "memory");
+                   ::"r"(smem_u32(rows_s + ((size_t)b * th + r) * pitch)), "l"(src), "r"(row_bytes), "r"(bar) : "memory");
     }
-    s_cnt[3] += 1u;
+    s_cnt[3 + b] += 1u;
   };
+
   if (tid == 0) {
-    mbar_init(rows_full, 1);
-    for (int i = 0; i < 4; ++i) mbar_init(acc_ready0 + 8 * i, 1);                   // tcgen05.commit
+    for (int b = 0; b < ROWBUFS; ++b) mbar_init(rows_full0 + 8 * b, 1);
+    for (int b = 0; b < ABUFS; ++b) {
+      mbar_init(a_full0 + 8 * b, GATHER_WARPS);
+      mbar_init(a_free0 + 8 * b, 1);
+    }
+    for (int s = 0; s < SLOTS; ++s) {
+      mbar_init(acc_ready0 + 8 * s, 1);
+      mbar_init(acc_free0 + 8 * s, COMPUTE_WARPS);
+    }
     *abort_flag = 0;
-    for (int i = 0; i < 4; ++i) s_cnt[i] = 0u;
+    for (int i = 0; i < 6; ++i) s_cnt[i] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     // the first rows travel while the CTA builds its tables
-    if ((int)blockIdx.x < p.groups) request_rows(blockIdx.x);
+    if ((int)blockIdx.x < p.groups)
+      for (uint32_t hs = 0; hs < (uint32_t)ROWBUFS; ++hs) request_half(hs);
   }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(p.tmem_cols) : "memory");
+  if (warp == MMA_WARP) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // H_128 as the B operand: B[n][k] = (-1)^popcount(n & k), K-major, 128-byte swizzle (the matrix is symmetric)
@@ -132,10 +169,21 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const uint32_t chunk = (uint32_t)((k0 & 63) >> 3);
     *reinterpret_cast<uint4*>(smem + OFF_H + (k0 >> 6) * ATOM + n * 128 + ((chunk ^ (n & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
   }
-  for (int i = tid; i < WARPS * 16; i += THREADS) s_part[i] = 0.f;
-  if (TAB_SMEM) {
-    for (int i = tid; i < p.dim; i += THREADS) s_table[(i >> 7) * TAB_PITCH + (i & 127)] = __ldg(p.offset + i);
-    for (int i = tid; i < p.dim / 2; i += THREADS) s_mask[(i >> 6) * MSK_PITCH + (i & 63)] = __ldg(p.posmask + i);
+  for (int i = tid; i < 2 * COMPUTE_WARPS * 16; i += THREADS) s_part[i] = 0.f;
+  if (TAB == 1) {
+    // 16 bytes per thread and load: one or two loads per thread, all in flight together
+    const uint4* src = reinterpret_cast<const uint4*>(p.offset);
+    for (int i = tid; i < p.dim / 4; i += THREADS)
+      reinterpret_cast<uint4*>(s_table)[(i >> 5) * (TAB_PITCH / 4) + (i & 31)] = __ldg(src + i);
+    const uint4* msrc = reinterpret_cast<const uint4*>(p.posmask);
+    for (int i = tid; i < p.dim / 8; i += THREADS)
+      reinterpret_cast<uint4*>(s_mask)[(i >> 4) * (MSK_PITCH / 4) + (i & 15)] = __ldg(msrc + i);
+  } else if (TAB == 2) {
+    const uint4* src = reinterpret_cast<const uint4*>(p.offset);
+    for (int i = tid; i < p.dim / 4; i += THREADS) {      // 4 offsets -> 2 words of the 16-bit table
+      const uint4 o = __ldg(src + i);
+      reinterpret_cast<uint2*>(s_table)[(i >> 5) * (MSK_PITCH / 2) + (i & 31)] = make_uint2(o.x | (o.y << 16), o.z | (o.w << 16));
+    }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -143,126 +191,156 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
 
-
-  const int q = warp & 3, kq = warp >> 2;          // tensor-memory lane quarter, column quarter
-  const int r = q * 32 + lane;                     // row of the operand tile = tensor-memory lane
-  // (token, block) pair of that row.  For T = 16 bits 3 and 5 of the row number trade places, so that a warp
-  // holds 8 tokens x 4 blocks: rows are 16-byte aligned in shared memory, tokens t and t + 8 share banks.
-  const int rp = (p.tshift == 4) ? ((r & ~0x28) | ((r & 8) << 2) | ((r & 32) >> 2)) : r;
-  const int t = rp & (T - 1);
-  const int j0 = rp >> p.tshift, jstep = H >> p.tshift;
-  const unsigned char* rowbytes = rows_s + (size_t)t * pitch;
-  const uint32_t a_row = (uint32_t)r * 128u;
-  const uint32_t sw = (uint32_t)(r & 7);
-  const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
-  const float inv_sqrt_h = rsqrtf((float)H);
-  const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kq * 32);
-  const uint64_t desc_h = smem_desc(smem_u32(smem + OFF_H));
-
-  // ---- pieces of the gather of tile i: offsets of the thread's 32 coordinates ...
-  auto gather_offsets = [&](int i, uint32_t (&h)[32]) {
-    const int j = j0 + i * jstep;
-    const uint4* tab = reinterpret_cast<const uint4*>(TAB_SMEM ? s_table + j * TAB_PITCH + kq * 32 : p.offset + j * H + kq * 32);
-#pragma unroll
-    for (int e4 = 0; e4 < 8; ++e4) {
-      const uint4 o = TAB_SMEM ? tab[e4] : __ldg(tab + e4);
-      h[4 * e4] = o.x; h[4 * e4 + 1] = o.y; h[4 * e4 + 2] = o.z; h[4 * e4 + 3] = o.w;
-    }
-  };
-  // ... the 16-bit loads of chunk c (8 coordinates), in place of their offsets ...
-  auto gather_chunk_loads = [&](int c, uint32_t (&h)[32]) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) h[8 * c + e] = *reinterpret_cast<const unsigned short*>(rowbytes + h[8 * c + e]);
-  };
-  // ... and the sign masks, the pairing and the 16-byte store of chunk c into the swizzled tile.
-  auto gather_chunk_store = [&](int i, int c, const uint32_t (&h)[32]) {
-    const int j = j0 + i * jstep;
-    const uint4* msk = reinterpret_cast<const uint4*>(TAB_SMEM ? s_mask + j * MSK_PITCH + kq * 16 : p.posmask + j * (H / 2) + kq * 16);
-    const uint4 m = TAB_SMEM ? msk[c] : __ldg(msk + c);
-    uint4 o;
-    o.x = prmt(h[8 * c], h[8 * c + 1], 0x5410u) ^ m.x;
-    o.y = prmt(h[8 * c + 2], h[8 * c + 3], 0x5410u) ^ m.y;
-    o.z = prmt(h[8 * c + 4], h[8 * c + 5], 0x5410u) ^ m.z;
-    o.w = prmt(h[8 * c + 6], h[8 * c + 7], 0x5410u) ^ m.w;
-    unsigned char* abuf = smem + OFF_A + (i & 1) * TILE + (kq >> 1) * ATOM + a_row;
-    const uint32_t chunk = (uint32_t)((kq & 1) * 4 + c);
-    *reinterpret_cast<uint4*>(abuf + ((chunk ^ sw) << 4)) = o;
-  };
   auto warp_wait = [&](uint32_t bar, uint32_t parity, int code) {
     if (lane == 0) mbar_wait(bar, parity, abort_flag, p.status, code);
     __syncwarp();
   };
-  // This warp has taken everything it needs from the row buffer for group `grp`; the last warp to say so
-  // requests the rows of the CTA's next group.
-  auto rows_done = [&](int grp) {
-    __syncwarp();
-    if (lane == 0) {
-      __threadfence_block();
-      const unsigned int old = atomicAdd(&s_cnt[2], 1u);
-      if ((old & (WARPS - 1)) == WARPS - 1) {
-        const int nxt = grp + stride;
-        if (nxt < p.groups && !*abort_flag) request_rows(nxt);
-      }
-    }
-  };
-  // This warp has written its part of operand tile i and has read what it needed from accumulator i; the last
-  // warp to say so multiplies the tile by H_128 into accumulator i and commits to acc_ready[i].
-  auto tile_done = [&](int i) {
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) {
-      __threadfence_block();
-      const unsigned int old = atomicAdd(&s_cnt[i & 1], 1u);
-      if ((old & (WARPS - 1)) == WARPS - 1) {
-        __threadfence_block();
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        const uint32_t a_addr = smem_u32(smem + OFF_A + (i & 1) * TILE);
-#pragma unroll
-        for (int k4 = 0; k4 < 8; ++k4) {
-          const uint64_t da = smem_desc(a_addr + (k4 >> 2) * ATOM) + 2 * (k4 & 3);
-          const uint64_t db = desc_h + (uint64_t)((k4 >> 2) * (ATOM >> 4)) + 2 * (k4 & 3);
-          const uint32_t acc = k4 > 0 ? 1u : 0u;
-          asm volatile(
-              "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-              " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-              ::"r"(tmem + (uint32_t)i * 128u), "l"(da), "l"(db), "r"(IDESC), "r"(acc) : "memory");
-        }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(acc_ready0 + 8 * i) : "memory");
-      }
-    }
-  };
+  // Which pair row r of tile i holds: its half, its block, and whether the row is in use.  (q = r / 32.)
+  auto tile_half = [&](int i, int q) { return nt3 ? (i == 0 ? 0 : (i == 2 ? 1 : (q >> 1))) : i; };
+  auto tile_block = [&](int i, int r) { return ((nt3 && i == 1) ? 128 + (r & 63) : r) >> p.ths; };
+  auto tile_valid = [&](int i, int r) { return nt3 ? (i != 1 || (r & 63) < rem) : r < p.pairs; };
 
-  // prologue: the tiles of the CTA's first group
-  if ((int)blockIdx.x < p.groups) {
-    warp_wait(rows_full, 0u, WAIT_ROWS);
-    for (int i = 0; i < p.ntiles; ++i) {
-      if (i >= 2) warp_wait(acc_ready0 + 8 * (i - 2), 0u, WAIT_ACC);   // the tile buffer was read by the MMAs of tile i - 2
-      if (j0 + i * jstep < kblocks) {
-        uint32_t h[32];
-        gather_offsets(i, h);
+  if (warp == MMA_WARP) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint64_t desc_h = smem_desc(smem_u32(smem + OFF_H));
+      uint32_t n = 0;                               // tiles issued so far (operand buffer n & 1, accumulator n % 3)
+      for (int grp = blockIdx.x; grp < p.groups; grp += stride) {
+        for (int i = 0; i < p.ntiles; ++i, ++n) {
+          const uint32_t buf = n & 1u, slot = n % 3u, use = n / 3u;
+          mbar_wait(a_full0 + 8 * buf, (n >> 1) & 1u, abort_flag, p.status, WAIT_AFULL);
+          if (use > 0u) mbar_wait(acc_free0 + 8 * slot, (use - 1u) & 1u, abort_flag, p.status, WAIT_ACCFREE);
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_tmem = tmem + A_COL0 + buf * 64u;     // 8 columns (16 bf16) per K step
 #pragma unroll
-        for (int c = 0; c < 4; ++c) gather_chunk_loads(c, h);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) gather_chunk_store(i, c, h);
+          for (int k4 = 0; k4 < 8; ++k4) {
+            const uint64_t db = desc_h + (uint64_t)((k4 >> 2) * (ATOM >> 4)) + 2 * (k4 & 3);
+            const uint32_t acc = k4 > 0 ? 1u : 0u;
+            asm volatile(
+                "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                ::"r"(tmem + slot * 128u), "r"(a_tmem + 8u * k4), "l"(db), "r"(IDESC), "r"(acc) : "memory");
+          }
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(acc_ready0 + 8 * slot) : "memory");
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(a_free0 + 8 * buf) : "memory");
+        }
       }
-      if (i == p.ntiles - 1) rows_done(blockIdx.x);
-      tile_done(i);
     }
-  }
-  int it = 0;
-  for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it) {
-    const int row0 = grp * T;
-    const uint32_t par = (uint32_t)it & 1u;
-    // ---------------- pass 1: squared norms from the rotated values ----------------
-    float ssq = 0.f;
-    for (int i = 0; i < p.ntiles; ++i) {
-      warp_wait(acc_ready0 + 8 * i, par, WAIT_ACC);
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      uint32_t v[32];
-      tmem_load32(tmem_thr + (uint32_t)i * 128u, v);
-      if (j0 + i * jstep < kblocks) {
+  } else if (warp >= COMPUTE_WARPS) {
+    // ------------------------------- gather warps -------------------------------
+    const int gw = warp - COMPUTE_WARPS;
+    const int gq = gw & 3, kh = gw >> 2;              // lane quarter of the tile, half of the 128 coordinates
+    const int r = gq * 32 + lane;                     // row of the operand tile
+    const int tl = lane & (th - 1);                   // token within its half (the same in every tile)
+    const uint32_t a_thr = tmem + ((uint32_t)(gq * 32) << 16) + A_COL0 + (uint32_t)kh * 32u;   // + 64 * buffer
+    uint32_t n = 0;
+    int it = 0;
+    for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it) {
+      for (int i = 0; i < p.ntiles; ++i, ++n) {
+        const uint32_t buf = n & 1u;
+        const int half = tile_half(i, gq), j = tile_block(i, r);
+        const uint32_t hs = 2u * (uint32_t)it + (uint32_t)half, rb = hs % 3u;
+        warp_wait(rows_full0 + 8 * rb, (hs / 3u) & 1u, WAIT_ROWS);
+        if (n >= 2u) warp_wait(a_free0 + 8 * buf, ((n >> 1) - 1u) & 1u, WAIT_AFREE);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        uint32_t w[32];
+        if (tile_valid(i, r)) {
+          const unsigned char* rowbytes = rows_s + ((size_t)rb * th + tl) * pitch;
+          // offsets of the thread's 64 coordinates, then the 64 loads (all in flight together), then masks and
+          // pairing: 32 words of two bf16, the thread's half row of the operand tile
+          if constexpr (TAB == 2) {
+            // two rounds of 32 coordinates: 16-bit offsets from shared memory, masks from global memory (requested
+            // before the gather loads so that their latency overlaps)
+#pragma unroll
+            for (int rd = 0; rd < 2; ++rd) {
+              uint32_t h[32];
+              const uint4* tab = reinterpret_cast<const uint4*>(s_table + j * MSK_PITCH + kh * 32 + rd * 16);
+#pragma unroll
+              for (int e8 = 0; e8 < 4; ++e8) {
+                const uint4 o = tab[e8];
+                h[8 * e8] = o.x & 0xFFFFu; h[8 * e8 + 1] = o.x >> 16; h[8 * e8 + 2] = o.y & 0xFFFFu; h[8 * e8 + 3] = o.y >> 16;
+                h[8 * e8 + 4] = o.z & 0xFFFFu; h[8 * e8 + 5] = o.z >> 16; h[8 * e8 + 6] = o.w & 0xFFFFu; h[8 * e8 + 7] = o.w >> 16;
+              }
+              const uint4* msk = reinterpret_cast<const uint4*>(p.posmask + j * (H / 2) + kh * 32 + rd * 16);
+              uint4 m[4];
+#pragma unroll
+              for (int c = 0; c < 4; ++c) m[c] = __ldg(msk + c);
+#pragma unroll
+              for (int e = 0; e < 32; ++e) h[e] = *reinterpret_cast<const unsigned short*>(rowbytes + h[e]);
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                w[16 * rd + 4 * c] = prmt(h[8 * c], h[8 * c + 1], 0x5410u) ^ m[c].x;
+                w[16 * rd + 4 * c + 1] = prmt(h[8 * c + 2], h[8 * c + 3], 0x5410u) ^ m[c].y;
+                w[16 * rd + 4 * c + 2] = prmt(h[8 * c + 4], h[8 * c + 5], 0x5410u) ^ m[c].z;
+                w[16 * rd + 4 * c + 3] = prmt(h[8 * c + 6], h[8 * c + 7], 0x5410u) ^ m[c].w;
+              }
+            }
+          } else {
+            uint32_t h[64];
+            const uint4* tab = reinterpret_cast<const uint4*>(TAB == 1 ? s_table + j * TAB_PITCH + kh * 64 : p.offset + j * H + kh * 64);
+#pragma unroll
+            for (int e4 = 0; e4 < 16; ++e4) {
+              const uint4 o = TAB == 1 ? tab[e4] : __ldg(tab + e4);
+              h[4 * e4] = o.x; h[4 * e4 + 1] = o.y; h[4 * e4 + 2] = o.z; h[4 * e4 + 3] = o.w;
+            }
+#pragma unroll
+            for (int e = 0; e < 64; ++e) h[e] = *reinterpret_cast<const unsigned short*>(rowbytes + h[e]);
+            const uint4* msk = reinterpret_cast<const uint4*>(TAB == 1 ? s_mask + j * MSK_PITCH + kh * 32 : p.posmask + j * (H / 2) + kh * 32);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const uint4 m = TAB == 1 ? msk[c] : __ldg(msk + c);
+              w[4 * c] = prmt(h[8 * c], h[8 * c + 1], 0x5410u) ^ m.x;
+              w[4 * c + 1] = prmt(h[8 * c + 2], h[8 * c + 3], 0x5410u) ^ m.y;
+              w[4 * c + 2] = prmt(h[8 * c + 4], h[8 * c + 5], 0x5410u) ^ m.z;
+              w[4 * c + 3] = prmt(h[8 * c + 6], h[8 * c + 7], 0x5410u) ^ m.w;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) w[c] = 0u;
+        }
+        // the operand tile lives in tensor memory: 32 columns of this thread's lane
+        tmem_store32(a_thr + buf * 64u, w);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        // the last gather warp to finish with a row buffer requests the half group that reuses it
+        const bool last0 = nt3 ? i == 1 : i == 0, last1 = i == p.ntiles - 1;
+        __syncwarp();
+        if (lane == 0) {
+          if (last0 || last1) {
+            __threadfence_block();
+            const uint32_t hsr = 2u * (uint32_t)it + (last1 ? 1u : 0u), b = hsr % 3u;
+            const unsigned int old = atomicAdd(&s_cnt[b], 1u);
+            if ((old & (GATHER_WARPS - 1)) == GATHER_WARPS - 1 && !*abort_flag) {
+              const long long g3 = (long long)blockIdx.x + (long long)((hsr + 3u) >> 1) * stride;
+              if (g3 < p.groups) request_half(hsr + 3u);
+            }
+          }
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_full0 + 8 * buf) : "memory");
+        }
+      }
+    }
+  } else {
+    // ------------------------------- compute warps -------------------------------
+    const int q = warp & 3, kq = warp >> 2;          // tensor-memory lane quarter, column quarter
+    const int r = q * 32 + lane;                     // row of the tile = tensor-memory lane
+    const int tl = lane & (th - 1);
+    const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
+    const float inv_sqrt_h = rsqrtf((float)H);
+    const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kq * 32);
+    uint32_t n0 = 0;                                  // sequence number of the group's first tile
+    int it = 0;
+    for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it, n0 += (uint32_t)p.ntiles) {
+      const int row0 = grp * T;
+      // ---------------- pass 1: sums of squares of the rotated values, per half ----------------
+      float ssq0 = 0.f, ssq1 = 0.f;
+      for (int i = 0; i < p.ntiles; ++i) {
+        const uint32_t n = n0 + (uint32_t)i, slot = n % 3u;
+        warp_wait(acc_ready0 + 8 * slot, (n / 3u) & 1u, WAIT_ACC);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        uint32_t v[32];
+        tmem_load32(tmem_thr + slot * 128u, v);
         unsigned long long acc2 = 0ull;
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
@@ -271,105 +349,68 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
         }
         float a0, a1;
         unpack2(acc2, a0, a1);
-        ssq += a0 + a1;
+        const float a = tile_valid(i, r) ? a0 + a1 : 0.f;
+        if (tile_half(i, q)) ssq1 += a; else ssq0 += a;
       }
-    }
-    // lanes of the warp that hold the same token add up; the lowest of them publishes the warp's partial sum
-    bool leader = true;
+      // lanes of the warp that hold the same token add up (they differ in the lane bits above log2 th) ...
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) {
-      const float other = __shfl_xor_sync(0xffffffffu, ssq, o);
-      const int ot = __shfl_xor_sync(0xffffffffu, t, o);
-      if (ot == t) {
-        ssq += other;
-        if (lane & o) leader = false;
+      for (int o = 16; o >= 1; o >>= 1)
+        if (o >= th) {
+          ssq0 += __shfl_xor_sync(0xffffffffu, ssq0, o);
+          ssq1 += __shfl_xor_sync(0xffffffffu, ssq1, o);
+        }
+      float* part = s_part + (it & 1) * (COMPUTE_WARPS * 16);
+      if (lane < th) {
+        part[warp * 16 + lane] = ssq0;
+        part[warp * 16 + 8 + lane] = ssq1;
       }
-    }
-    if (leader) s_part[warp * 16 + t] = ssq;
-    __syncthreads();
-    float tot = 0.f;
+      asm volatile("bar.sync 1, %0;" ::"n"(COMPUTE_THREADS) : "memory");
+      // ... and the 16 warps' partial sums in a fixed order: lane L adds 8 warps for slot L & 15
+      float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < WARPS; ++w) tot += s_part[w * 16 + t];
-    const float s = sqrtf(tot * (1.0f / (float)H));
-    const bool row_ok = row0 + t < p.rows;
-    // warps 0 and 1 (lane quarters 0 and 1, column quarter 0) hold every token between them
-    if (warp == ((p.tshift == 4) ? (t >> 3) : 0) && leader && row_ok) {
-      if (p.bf16_norm) reinterpret_cast<__nv_bfloat16*>(p.out_norm)[row0 + t] = __float2bfloat16_rn(s);
-      else reinterpret_cast<float*>(p.out_norm)[row0 + t] = s;
-    }
-    // ---------------- pass 2 of this group, fused with the gather of the CTA's next group ----------------
-    // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
-    const float kappa = 1.0f / (sqrtf((float)H) * (s + 1e-10f) * p.poly.clamp);
-    const int nxt = grp + stride;
-    const bool has_next = nxt < p.groups;
-    const uint32_t npar = par ^ 1u;
-    if (has_next) warp_wait(rows_full, npar, WAIT_ROWS);
-    for (int i = 0; i < p.ntiles; ++i) {
-      const int j = j0 + i * jstep;
-      const bool pair_ok = j < kblocks;
-      const bool gat = has_next && pair_ok;
-      if (has_next && i >= 2) warp_wait(acc_ready0 + 8 * (i - 2), npar, WAIT_ACC);
-      uint32_t h[32];
-      if (gat) {
-        gather_offsets(i, h);
-        gather_chunk_loads(0, h);
-        gather_chunk_loads(1, h);
-      }
-      uint32_t vb[32];
-      tmem_load32(tmem_thr + (uint32_t)i * 128u, vb);
-      float v[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(vb[e]);
-      const bool out_ok = pair_ok && row_ok;
-      if (p.dbg != nullptr && out_ok) {
-        float* d = p.dbg + (size_t)(row0 + t) * p.dim + j * H + kq * 32;
-#pragma unroll
-        for (int e = 0; e < 32; ++e) d[e] = v[e] * inv_sqrt_h;
-      }
-      uint32_t words[BITS];
-      if constexpr (BITS == 4) {
-        // The gather sits in the first half of the tile: chunks 2 and 3 are loaded before word 0 is packed and
-        // stored before word 1, so every shared-memory load has a level search between its issue and its use,
-        // and the tile is handed over (and its MMAs start) while words 1 to 3 are still being packed.
-        if (gat) {
-          gather_chunk_loads(2, h);
-          gather_chunk_loads(3, h);
-          gather_chunk_store(i, 0, h);
-          gather_chunk_store(i, 1, h);
-        }
-        words[0] = pack8_4bit(v, kappa, poly);
-        if (gat) {
-          gather_chunk_store(i, 2, h);
-          gather_chunk_store(i, 3, h);
-        }
-        if (has_next) {
-          if (i == p.ntiles - 1) rows_done(nxt);
-          tile_done(i);
-        }
-#pragma unroll
-        for (int c = 1; c < 4; ++c) words[c] = pack8_4bit(v + 8 * c, kappa, poly);
-      } else {
-        if (gat) {
-          gather_chunk_loads(2, h);
-          gather_chunk_loads(3, h);
-        }
-        pack32<BITS>(v, kappa, poly, words);
-        if (gat) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) gather_chunk_store(i, c, h);
-        }
-        if (has_next) {
-          if (i == p.ntiles - 1) rows_done(nxt);
-          tile_done(i);
+      for (int w = 0; w < 8; ++w) tot += part[((lane >> 4) * 8 + w) * 16 + (lane & 15)];
+      tot += __shfl_xor_sync(0xffffffffu, tot, 16);
+      const float nrm = sqrtf(tot * (1.0f / (float)H));            // of slot lane & 15 = (half, token)
+      if (warp == 0 && lane < 16 && (lane & 7) < th) {
+        const int row = row0 + (lane >> 3) * th + (lane & 7);
+        if (row < p.rows) {
+          if (p.bf16_norm) reinterpret_cast<__nv_bfloat16*>(p.out_norm)[row] = __float2bfloat16_rn(nrm);
+          else reinterpret_cast<float*>(p.out_norm)[row] = nrm;
         }
       }
-      if (out_ok) {
-        uint32_t* dst = p.out_idx + (size_t)(row0 + t) * p.pitch_words + (j * (H / 32) + kq) * BITS;
-        if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
-        else if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(words[0], words[1]);
-        else {
+      const float s0 = __shfl_sync(0xffffffffu, nrm, tl), s1 = __shfl_sync(0xffffffffu, nrm, 8 + tl);
+      // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
+      const float kappa0 = 1.0f / (sqrtf((float)H) * (s0 + 1e-10f) * p.poly.clamp);
+      const float kappa1 = 1.0f / (sqrtf((float)H) * (s1 + 1e-10f) * p.poly.clamp);
+      // ---------------- pass 2: level search and packing ----------------
+      for (int i = 0; i < p.ntiles; ++i) {
+        const uint32_t n = n0 + (uint32_t)i, slot = n % 3u;
+        const int half = tile_half(i, q), j = tile_block(i, r);
+        uint32_t vb[32];
+        tmem_load32(tmem_thr + slot * 128u, vb);
+        // the accumulator may be overwritten as soon as every compute warp has read it
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_free0 + 8 * slot) : "memory");
+        const int row = row0 + half * th + tl;
+        if (tile_valid(i, r) && row < p.rows) {
+          float v[32];
 #pragma unroll
-          for (int c = 0; c < BITS; ++c) dst[c] = words[c];
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(vb[e]);
+          if (p.dbg != nullptr) {
+            float* d = p.dbg + (size_t)row * p.dim + j * H + kq * 32;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) d[e] = v[e] * inv_sqrt_h;
+          }
+          uint32_t words[BITS];
+          pack32<BITS>(v, half ? kappa1 : kappa0, poly, words);
+          uint32_t* dst = p.out_idx + (size_t)row * p.pitch_words + (j * (H / 32) + kq) * BITS;
+          if constexpr (BITS == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
+          else if constexpr (BITS == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(words[0], words[1]);
+          else {
+#pragma unroll
+            for (int c = 0; c < BITS; ++c) dst[c] = words[c];
+          }
         }
       }
     }
@@ -378,10 +419,15 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   // after a wait gave up somewhere, a requested copy may still be in flight: let it land before the CTA ends
-  if (tid == 0 && *abort_flag && s_cnt[3] > 0u) mbar_wait(rows_full, (s_cnt[3] - 1u) & 1u, abort_flag, p.status, WAIT_DRAIN);
-  if (warp == 0) {
+  if (tid == 0 && *abort_flag) {
+    int keep_waiting = 0;      // (the CTA's abort flag is already up: it must not cut this wait short)
+    for (int b = 0; b < ROWBUFS; ++b)
+      if (s_cnt[3 + b] > 0u)
+        mbar_wait(rows_full0 + 8 * b, (s_cnt[3 + b] - 1u) & 1u, &keep_waiting, p.status, WAIT_DRAIN, 200000000ll);
+  }
+  if (warp == MMA_WARP) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TMEM_COLS) : "memory");
   }
 }
 
