@@ -341,15 +341,18 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         uint32_t v[32];
         tmem_load32(tmem_thr + slot * 128u, v);
-        unsigned long long acc2 = 0ull;
+        unsigned long long qa = 0ull, qb = 0ull;      // two chains, fixed order
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const unsigned long long x2 = pack2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-          acc2 = fma2(x2, x2, acc2);
+        for (int e = 0; e < 16; e += 2) {
+          const unsigned long long xa = pack2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+          const unsigned long long xb = pack2(__uint_as_float(v[2 * e + 2]), __uint_as_float(v[2 * e + 3]));
+          qa = fma2(xa, xa, qa);
+          qb = fma2(xb, xb, qb);
         }
-        float a0, a1;
-        unpack2(acc2, a0, a1);
-        const float a = tile_valid(i, r) ? a0 + a1 : 0.f;
+        float a0, a1, b0, b1;
+        unpack2(qa, a0, a1);
+        unpack2(qb, b0, b1);
+        const float a = tile_valid(i, r) ? (a0 + a1) + (b0 + b1) : 0.f;
         if (tile_half(i, q)) ssq1 += a; else ssq0 += a;
       }
       // lanes of the warp that hold the same token add up (they differ in the lane bits above log2 th) ...
