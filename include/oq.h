@@ -184,6 +184,15 @@ int oq_device_status(int* status);
  * OQ_ERR_DEVICE_TIMEOUT with *status == 9 and leave the word clear again. */
 int oq_selftest_bounded_wait(void* stream);
 
+/* Host-only query (no device needed): which kernel oq_rotate_quantize_act / oq_quantize_weights would launch for
+ * this rotation and codebook, and its shape: *kernel = 1 general, 2 register butterflies, 3 tensor cores;
+ * *rows_per_group = rows one CTA holds in shared memory at a time (1 for the general kernel);
+ * *tiles_per_group = 128-row tensor-core tiles per group (0 for the other kernels); *smem_bytes = dynamic shared
+ * memory per CTA.  Any output pointer may be NULL.  Honours oq_debug_select_rq_kernel.  Returns OQ_OK,
+ * OQ_ERR_INVALID_ARG (NULL handle, dims differ) or OQ_ERR_UNSUPPORTED (dim not a multiple of 128). */
+int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows_per_group, int* tiles_per_group,
+               size_t* smem_bytes);
+
 /* Test helper: selects the kernel behind oq_rotate_quantize_act / oq_quantize_weights for the following calls of
  * this process: 0 = choose by shape (default), 1 = general kernel (any block size; butterflies in shared memory),
  * 2 = register-butterfly kernel (blocks of 64, 128, 256), 3 = tensor-core kernel (blocks of 128; the block

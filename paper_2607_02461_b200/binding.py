@@ -50,6 +50,7 @@ def lib():
             "oq_device_status": (i, [C.POINTER(i)]),
             "oq_selftest_bounded_wait": (i, [vp]),
             "oq_debug_select_rq_kernel": (i, [i]),
+            "oq_rq_plan": (i, [vp, vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(sz)]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
         for name, (res, args) in sig.items():
@@ -215,6 +216,13 @@ def oq_device_status():
 
 def oq_selftest_bounded_wait():
     _check(lib().oq_selftest_bounded_wait(_stream()))
+
+
+def oq_rq_plan(rot, cb):
+    """(kernel, rows_per_group, tiles_per_group, smem_bytes) of the rotate+quantize launch for these handles."""
+    k, r, t, m = C.c_int(0), C.c_int(0), C.c_int(0), C.c_size_t(0)
+    _check(lib().oq_rq_plan(rot.handle, cb.handle, C.byref(k), C.byref(r), C.byref(t), C.byref(m)))
+    return k.value, r.value, t.value, m.value
 
 
 def oq_debug_select_rq_kernel(which):

@@ -326,6 +326,28 @@ int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, c
                                     stream);
 }
 
+int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows_per_group, int* tiles_per_group,
+               size_t* smem_bytes) {
+  if (!rot || !cb) return fail(OQ_ERR_INVALID_ARG, "oq_rq_plan: NULL handle");
+  if (rot->dim != cb->dim) return fail(OQ_ERR_INVALID_ARG, "oq_rq_plan: dim differs between the rotation and the codebook");
+  if (rot->dim % 128) return fail(OQ_ERR_UNSUPPORTED, "oq_rq_plan: dim must be a multiple of 128");
+  int k = 1, rows = 1, tiles = 0;
+  size_t smem = (size_t)rot->dim * 5;
+  TcPlan tp;
+  FastPlan fp;
+  const bool tc_ok = plan_tc(rot->dim, rot->block, cb, &tp);
+  if ((g_forced_kernel == 0 && tc_ok && tp.fill >= 0.6) || (g_forced_kernel == 3 && tc_ok)) {
+    k = 3; rows = 2 << tp.ths; tiles = tp.ntiles; smem = tp.smem;
+  } else if (g_forced_kernel != 1 && plan_fast(rot->dim, rot->block, cb, &fp)) {
+    k = 2; rows = fp.T; smem = fp.smem;
+  }
+  if (kernel) *kernel = k;
+  if (rows_per_group) *rows_per_group = rows;
+  if (tiles_per_group) *tiles_per_group = tiles;
+  if (smem_bytes) *smem_bytes = smem;
+  return OQ_OK;
+}
+
 int oq_debug_select_rq_kernel(int which) {
   if (which < 0 || which > 3) return fail(OQ_ERR_INVALID_ARG, "oq_debug_select_rq_kernel: which must be 0..3");
   g_forced_kernel = which;

@@ -121,3 +121,26 @@ def test_level_search_polynomial_counts_boundaries(dim, bits):
         if bad.any():
             dist = np.min(np.abs(texact[bad][:, None] - beta[None, :]), axis=1)
             assert dist.max() <= 1e-6 * beta[-1] and np.abs(mag - want)[bad].max() == 1
+
+
+@pytest.mark.parametrize("dim,block,kernel,rows,tiles", [
+    (3072, 128, 3, 16, 3),      # FLUX hidden size: 8 tokens per half group, 192 (token, block) pairs per half
+    (12288, 128, 3, 4, 3),      # FLUX MLP width
+    (5120, 128, 3, 8, 3),       # Wan hidden size: 160 pairs per half
+    (13824, 128, 3, 2, 2),      # Wan FFN width: 108 pairs per half, one tile per half
+    (1024, 128, 2, 16, 0),      # 64 pairs per half would fill half of the tiles: register kernel
+    (3072, 64, 2, 16, 0),
+    (3072, 256, 2, 8, 0),
+    (3072, 1024, 1, 1, 0),      # the paper's default block for this width: general kernel
+])
+def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
+    """Host-side launch planning (no device needed): kernel choice and group shape for the benchmark widths."""
+    rot, cb = B.oq_make_rpbh(dim, block, 0), B.oq_build_codebook(dim, 4)
+    k, r, t, smem = B.oq_rq_plan(rot, cb)
+    assert (k, r, t) == (kernel, rows, tiles)
+    assert smem <= 227 * 1024
+    B.oq_debug_select_rq_kernel(1)
+    try:
+        assert B.oq_rq_plan(rot, cb)[0] == 1
+    finally:
+        B.oq_debug_select_rq_kernel(0)
