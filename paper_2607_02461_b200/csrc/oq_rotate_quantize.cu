@@ -198,7 +198,7 @@ struct TcPlan {
   double fill;      // used rows of the operand tiles / all rows
 };
 static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
-  if (block != 128 || !cb->poly.ok) return false;
+  if ((block != 64 && block != 128 && block != 256) || !cb->poly.ok) return false;
   const size_t kMaxSmem = 227 * 1024;
   const int kblocks = dim / 128;
   for (int ths = 3; ths >= 0; --ths) {
@@ -223,13 +223,19 @@ static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
   return false;
 }
 
-template <int BITS>
+template <int BITS, int BLK>
 static cudaError_t launch_tc_bits(int tab, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
-  auto k = tab == 1 ? rq_tc_kernel<BITS, 1> : tab == 2 ? rq_tc_kernel<BITS, 2> : rq_tc_kernel<BITS, 0>;
+  auto k = tab == 1 ? rq_tc_kernel<BITS, 1, BLK> : tab == 2 ? rq_tc_kernel<BITS, 2, BLK> : rq_tc_kernel<BITS, 0, BLK>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   k<<<grid, rqtc::THREADS, smem, st>>>(prm);
   return cudaGetLastError();
+}
+template <int BITS>
+static cudaError_t launch_tc_block(int block, int tab, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
+  if (block == 64) return launch_tc_bits<BITS, 64>(tab, grid, smem, st, prm);
+  if (block == 256) return launch_tc_bits<BITS, 256>(tab, grid, smem, st, prm);
+  return launch_tc_bits<BITS, 128>(tab, grid, smem, st, prm);
 }
 
 template <bool kBf16Norm>
@@ -263,9 +269,9 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
     prm.bf16_norm = kBf16Norm ? 1 : 0;
     prm.status = status;
     int grid = sms < prm.groups ? sms : prm.groups;
-    if (cb->bits == 4) e = launch_tc_bits<4>(tp.tab, grid, tp.smem, st, prm);
-    else if (cb->bits == 3) e = launch_tc_bits<3>(tp.tab, grid, tp.smem, st, prm);
-    else e = launch_tc_bits<2>(tp.tab, grid, tp.smem, st, prm);
+    if (cb->bits == 4) e = launch_tc_block<4>(rot->block, tp.tab, grid, tp.smem, st, prm);
+    else if (cb->bits == 3) e = launch_tc_block<3>(rot->block, tp.tab, grid, tp.smem, st, prm);
+    else e = launch_tc_block<2>(rot->block, tp.tab, grid, tp.smem, st, prm);
     if (e != cudaSuccess) return cuda_fail(e, fn);
     return OQ_OK;
   }

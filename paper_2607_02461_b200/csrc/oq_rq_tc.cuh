@@ -1,4 +1,4 @@
-// Fused rotate+quantize kernel for Hadamard blocks of 128 with the block transform on the tensor cores.
+// Fused rotate+quantize kernel for Hadamard blocks of 64, 128 and 256 with the block transform on the tensor cores.
 //
 // The rotation of Eq. 7 / Eq. 4 is  z = blkdiag(H_128 D_j) P x : a gather, a sign flip and, per block of 128
 // rotated coordinates, a product with the 128 x 128 matrix of +-1.  Butterflies in registers cost ~6
@@ -6,7 +6,8 @@
 // as bf16 into a shared-memory operand tile instead and one tcgen05.mma per 16 coordinates multiplies 128
 // (token, block) pairs by H_128 (entries +-1 are exact in bf16, the inputs are bf16 already, the sums are
 // accumulated in fp32 in tensor memory).  The rest of the path reads tensor memory twice: once for the row
-// norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.
+// norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.  Blocks of 64 use a block-diagonal
+// operand (two blocks per 128 coordinates); blocks of 256 add one butterfly stage across two tile rows.
 //
 // Work units.  A group is 2 th consecutive rows (th = 1, 2, 4 or 8 tokens per HALF group, chosen so that the
 // P = th * dim / 128 (token, block) pairs of a half number at most 192).  Each half has its own row buffer and
@@ -82,7 +83,8 @@ __host__ __device__ constexpr uint32_t row_pitch_bytes(int dim) { return 2u * (u
 
 // TAB: where the gather tables live.  0: global memory (read-only path); 1: both copied to shared memory (32-bit
 // offsets, masks); 2: offsets copied to shared memory as 16-bit values, masks stay in global memory.
-template <int BITS, int TAB>
+// BLK: the Hadamard block, 64, 128 or 256 (256: one butterfly stage across two tile rows after the tensor-core product).
+template <int BITS, int TAB, int BLK>
 __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParams p) {
   using namespace rqtc;
   extern __shared__ unsigned char smem_dyn[];
@@ -156,14 +158,21 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // H_128 as the B operand: B[n][k] = (-1)^popcount(n & k), K-major, 128-byte swizzle (the matrix is symmetric)
+  // The B operand, K-major, 128-byte swizzle: H_128 with B[n][k] = (-1)^popcount(n & k) (symmetric) for blocks of 128
+  // and 256, blkdiag(H_64, H_64) for blocks of 64.
   for (int c = tid; c < 128 * 16; c += THREADS) {
     const int n = c >> 4, k0 = (c & 15) * 8;
     uint32_t w[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const uint32_t lo = (__popc(n & (k0 + 2 * e)) & 1) ? 0xBF80u : 0x3F80u;
-      const uint32_t hi = (__popc(n & (k0 + 2 * e + 1)) & 1) ? 0xBF80u : 0x3F80u;
+      const int ka = k0 + 2 * e, kb2 = ka + 1;
+      constexpr int hm = BLK == 64 ? 63 : 127;       // index bits inside one Hadamard block of the tile row
+      uint32_t lo = (__popc(n & ka & hm) & 1) ? 0xBF80u : 0x3F80u;
+      uint32_t hi = (__popc(n & kb2 & hm) & 1) ? 0xBF80u : 0x3F80u;
+      if (BLK == 64) {           // two independent blocks of 64 per tile row: blkdiag(H_64, H_64)
+        if ((n ^ ka) & 64) lo = 0u;
+        if ((n ^ kb2) & 64) hi = 0u;
+      }
       w[e] = lo | (hi << 16);
     }
     const uint32_t chunk = (uint32_t)((k0 & 63) >> 3);
@@ -327,7 +336,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const int r = q * 32 + lane;                     // row of the tile = tensor-memory lane
     const int tl = lane & (th - 1);
     const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
-    const float inv_sqrt_h = rsqrtf((float)H);
+    const float inv_sqrt_h = rsqrtf((float)BLK);
+    constexpr float mma_h = BLK < H ? (float)BLK : (float)H;   // the tensor-core product multiplies squared norms by this
     const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kq * 32);
     uint32_t n0 = 0;                                  // sequence number of the group's first tile
     int it = 0;
@@ -373,7 +383,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
 #pragma unroll
       for (int w = 0; w < 8; ++w) tot += part[((lane >> 4) * 8 + w) * 16 + (lane & 15)];
       tot += __shfl_xor_sync(0xffffffffu, tot, 16);
-      const float nrm = sqrtf(tot * (1.0f / (float)H));            // of slot lane & 15 = (half, token)
+      const float nrm = sqrtf(tot * (1.0f / mma_h));               // of slot lane & 15 = (half, token)
       if (warp == 0 && lane < 16 && (lane & 7) < th) {
         const int row = row0 + (lane >> 3) * th + (lane & 7);
         if (row < p.rows) {
@@ -383,8 +393,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
       }
       const float s0 = __shfl_sync(0xffffffffu, nrm, tl), s1 = __shfl_sync(0xffffffffu, nrm, 8 + tl);
       // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
-      const float kappa0 = 1.0f / (sqrtf((float)H) * (s0 + 1e-10f) * p.poly.clamp);
-      const float kappa1 = 1.0f / (sqrtf((float)H) * (s1 + 1e-10f) * p.poly.clamp);
+      const float kappa0 = 1.0f / (sqrtf((float)BLK) * (s0 + 1e-10f) * p.poly.clamp);
+      const float kappa1 = 1.0f / (sqrtf((float)BLK) * (s1 + 1e-10f) * p.poly.clamp);
       // ---------------- pass 2: level search and packing ----------------
       for (int i = 0; i < p.ntiles; ++i) {
         const uint32_t n = n0 + (uint32_t)i, slot = n % 3u;
@@ -395,6 +405,16 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_free0 + 8 * slot) : "memory");
+        if constexpr (BLK == 256) {
+          // H_256 = [[H_128, H_128], [H_128, -H_128]]: the two halves of a block sit th rows apart, in the same warp
+          const float sg = (lane & th) ? -1.f : 1.f;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float mine = __uint_as_float(vb[e]);
+            const float other = __shfl_xor_sync(0xffffffffu, mine, th);
+            vb[e] = __float_as_uint(fmaf(mine, sg, other));      // low half: mine + other; high half: other - mine
+          }
+        }
         const int row = row0 + half * th + tl;
         if (tile_valid(i, r) && row < p.rows) {
           float v[32];

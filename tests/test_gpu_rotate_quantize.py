@@ -92,6 +92,16 @@ def test_every_kernel_matches_oracle_on_blocks_of_128(d, n, bits, kernel):
     assert check_rows(xb, 128, 1, bits, kernel=kernel) <= 1e-4
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("block", [64, 256])
+@pytest.mark.parametrize("d,n", [(256, 40), (1024, 67), (3072, 67), (5120, 35), (12288, 21), (13824, 9)])
+def test_tensor_core_kernel_on_blocks_of_64_and_256(d, n, block, bits):
+    """Blocks of 64 are two independent transforms per 128-coordinate tile row (block-diagonal operand); blocks of
+    256 add one butterfly stage across the two tile rows of a block."""
+    xb = synth.activations(n, d, seed=1300 + bits)
+    assert check_rows(xb, block, 5, bits, kernel=TENSOR) <= 1e-4
+
+
 @pytest.mark.parametrize("kernel", [REGISTERS, TENSOR])
 def test_kernels_agree_with_each_other_on_many_groups(kernel):
     """More row groups than CTAs (several pipeline rounds per CTA), ragged last group: same packed words and

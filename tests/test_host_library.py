@@ -129,8 +129,9 @@ def test_level_search_polynomial_counts_boundaries(dim, bits):
     (5120, 128, 3, 8, 3),       # Wan hidden size: 160 pairs per half
     (13824, 128, 3, 2, 2),      # Wan FFN width: 108 pairs per half, one tile per half
     (1024, 128, 2, 16, 0),      # 64 pairs per half would fill half of the tiles: register kernel
-    (3072, 64, 2, 16, 0),
-    (3072, 256, 2, 8, 0),
+    (3072, 64, 3, 16, 3),       # blocks of 64 and 256 use the same 128-coordinate tile rows
+    (3072, 256, 3, 16, 3),
+    (1024, 256, 2, 8, 0),
     (3072, 1024, 1, 1, 0),      # the paper's default block for this width: general kernel
 ])
 def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
