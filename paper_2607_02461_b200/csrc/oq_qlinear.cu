@@ -194,19 +194,21 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
   // Two ways to split a stage's 128 rows x 128 coordinates among 256 threads:
   //  * 4-bit operands: thread = (row t2/2, 32-coordinate half t2%2) of BOTH 64-coordinate swizzle atoms: one
   //    16-byte load per piece, adjacent lanes read adjacent 16 bytes;
-  //  * 3- and 2-bit operands: thread = (row t2%128, atom t2/128), 64 contiguous coordinates: 24 / 16 bytes,
-  //    8- / 16-byte aligned, instead of 12- / 8-byte pieces.
+  //  * 3- and 2-bit operands: thread = (row t2/2, atom t2%2), 64 contiguous coordinates: 24 / 16 bytes, 8- / 16-byte
+  //    aligned, instead of 12- / 8-byte pieces; adjacent lanes read the two adjacent pieces of one row (whole
+  //    sectors per warp).  The thread of atom 1 handles its two 32-coordinate pieces in the opposite order.
   // Inside an atom row r occupies 128 bytes and its 16-byte chunk c sits at position c ^ (r & 7); both
-  // mappings give the 8 lanes of a quarter warp 8 different chunk positions, i.e. all 32 banks.
+  // mappings give the 8 lanes of a quarter warp 8 different chunk positions, i.e. all 32 banks (4 rows x 2
+  // lanes: the lanes of atom 0 store chunks q ^ r, those of atom 1 chunks (q + 4) ^ r at the same time).
   constexpr bool CONTIG = BITS != 4;
-  const int row = CONTIG ? (t2 & 127) : (t2 >> 1);
-  const int sub = CONTIG ? (t2 >> 7) : (t2 & 1);      // atom (CONTIG) or half of each atom
+  const int row = t2 >> 1;
+  const int sub = t2 & 1;                             // atom (CONTIG) or half of each atom
   const int pitch = dim / 32 * BITS;
   constexpr int WPA = 2 * BITS;                       // words per 64 coordinates of one row
   unsigned char* const tile0 = smem + (IS_A ? 0u : PA_BYTES) + (uint32_t)row * 128u + (CONTIG ? (uint32_t)sub * ATOM_BYTES : 0u);
   const uint32_t rx = (uint32_t)(row & 7) << 4;
-  const uint32_t c0b = CONTIG ? 0u : (uint32_t)sub * 64u;          // first chunk (in bytes) of the first piece
-  const uint32_t second = CONTIG ? 64u : ATOM_BYTES;                // where the second piece goes relative to it
+  const uint32_t c0b = CONTIG ? (uint32_t)sub * 64u : (uint32_t)sub * 64u;   // first chunk (in bytes) of the piece stored first
+  const uint32_t second = CONTIG ? (sub ? 0u : 64u) : ATOM_BYTES;    // where the other piece goes (CONTIG: chunk offset; else: atom)
   uint32_t st = 0, ph = 0;
   bool first_round = true;
   Raw<BITS> n0r, n1r;                                 // packed words of the NEXT stage
@@ -235,7 +237,7 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
   fetch_next();
   for (int tile = pair_id; tile < ntiles; tile += npairs) {
     for (int kb = 0; kb < kblocks; ++kb) {
-      const Raw<BITS> c0 = n0r, c1 = n1r;
+      const Raw<BITS> c0 = (CONTIG && sub) ? n1r : n0r, c1 = (CONTIG && sub) ? n0r : n1r;
       fetch_next();
       if (!first_round) {
         if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
