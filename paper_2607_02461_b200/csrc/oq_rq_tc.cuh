@@ -77,6 +77,7 @@ constexpr uint32_t TILE = 2 * ATOM;               // 128 rows x 128 bf16
 constexpr uint32_t OFF_H = 0, OFF_ROWS = TILE;
 constexpr int TAB_PITCH = 132, MSK_PITCH = 68;    // words per block of the shared-memory table copies
 constexpr int MAX_PAIRS = 192;
+constexpr unsigned GATHER_SLEEP_NS = 256;         // between polls of a gather warp that waits for an operand tile
 enum { WAIT_ROWS = 11, WAIT_AFULL = 12, WAIT_ACC = 13, WAIT_DRAIN = 14, WAIT_AFREE = 15, WAIT_ACCFREE = 16 };
 __host__ __device__ constexpr uint32_t row_pitch_bytes(int dim) { return 2u * (uint32_t)dim + 16u; }
 }  // namespace rqtc
@@ -251,7 +252,10 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
         const int half = tile_half(i, gq), j = tile_block(i, r);
         const uint32_t hs = 2u * (uint32_t)it + (uint32_t)half, rb = hs % 3u;
         warp_wait(rows_full0 + 8 * rb, (hs / 3u) & 1u, WAIT_ROWS);
-        if (n >= 2u) warp_wait(a_free0 + 8 * buf, ((n >> 1) - 1u) & 1u, WAIT_AFREE);
+        if (n >= 2u) {     // the gather runs ahead of the other warps: a long sleep between polls leaves them the issue slots
+          if (lane == 0) mbar_wait(a_free0 + 8 * buf, ((n >> 1) - 1u) & 1u, abort_flag, p.status, WAIT_AFREE, WAIT_CYCLES, GATHER_SLEEP_NS);
+          __syncwarp();
+        }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         uint32_t w[32];
         if (tile_valid(i, r)) {

@@ -28,12 +28,12 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // `code` in the global status word, raises the CTA's abort flag and returns; callers carry on to the
 // common tear-down so tensor memory is always released.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code, long long max_cycles = WAIT_CYCLES) {
+                                          int code, long long max_cycles = WAIT_CYCLES, unsigned sleep_ns = 32) {
   if (mbar_try(bar, parity)) return;
   const long long t0 = clock64();
   int polls = 0;
   while (!mbar_try(bar, parity)) {
-    __nanosleep(32);   // a waiting lane should not take issue slots from the warps it waits for
+    __nanosleep(sleep_ns);   // a waiting lane should not take issue slots from the warps it waits for
     if (*abort_flag) return;
     if ((++polls & 1023) == 0) {
       if (*reinterpret_cast<volatile int*>(status) != 0 || clock64() - t0 > max_cycles) {
