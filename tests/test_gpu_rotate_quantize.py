@@ -125,6 +125,37 @@ def test_kernels_agree_with_each_other_on_many_groups(kernel):
     assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 1e-4
 
 
+@pytest.mark.parametrize("n", [1, 2, 15, 16, 17, 31, 33])
+@pytest.mark.parametrize("d,block", [(3072, 128), (12288, 64), (5120, 256)])
+def test_tensor_core_kernel_with_few_rows_and_padded_rows(n, d, block):
+    """Fewer rows than one group, a ragged last group (also one whose second half is empty), and a leading dimension
+    larger than dim: same indices as the general kernel (flips only between neighbours, rarely), same norms, and the
+    all-zero row stays on the middle boundary."""
+    import torch
+    xb = synth.activations(n, d, seed=1400 + n)
+    if n > 2:
+        xb[n // 2, :] = 0
+    rot, cb = B.oq_make_rpbh(d, block, 4), B.oq_build_codebook(d, 4)
+    wide = torch.zeros((n, d + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :d] = _dev(xb)
+    B.oq_debug_select_rq_kernel(GENERAL)
+    ref_idx, ref_norm = B.oq_rotate_quantize_act(wide[:, :d], rot, cb)
+    B.oq_debug_select_rq_kernel(TENSOR)
+    assert B.oq_rq_plan(rot, cb)[0] == TENSOR
+    idx, norm = B.oq_rotate_quantize_act(wide[:, :d], rot, cb)
+    B.oq_debug_select_rq_kernel(AUTO)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.allclose(norm, ref_norm, rtol=2e-6, atol=0)
+    a = B.oq_unpack_indices(idx, n, d, 4).to(torch.int16)
+    b = B.oq_unpack_indices(ref_idx, n, d, 4).to(torch.int16)
+    diff = (a - b).abs()
+    assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 1e-4
+    if n > 2:
+        assert norm[n // 2].item() == 0.0
+        assert torch.all((a[n // 2] == 7) | (a[n // 2] == 8))
+
+
 def test_config1_single_linear_activation_side():
     xb = synth.activations(256, 1024, seed=1000)
     assert check_rows(xb, 128, 0, 4) <= 1e-5
