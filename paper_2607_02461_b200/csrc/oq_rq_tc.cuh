@@ -326,6 +326,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
             const uint32_t hsr = 2u * (uint32_t)it + (last1 ? 1u : 0u), b = hsr % 3u;
             const unsigned int old = atomicAdd(&s_cnt[b], 1u);
             if ((old & (GATHER_WARPS - 1)) == GATHER_WARPS - 1 && !*abort_flag) {
+              __threadfence_block();     // the other warps' reads of the buffer are ordered before the copies below
               const long long g3 = (long long)blockIdx.x + (long long)((hsr + 3u) >> 1) * stride;
               if (g3 < p.groups) request_half(hsr + 3u);
             }
