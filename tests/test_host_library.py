@@ -145,3 +145,17 @@ def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
         assert B.oq_rq_plan(rot, cb)[0] == 1
     finally:
         B.oq_debug_select_rq_kernel(0)
+
+
+def test_rotate_quantize_plan_rejects_mismatched_handles():
+    rot = B.oq_make_rpbh(1024, 128, 0)
+    with pytest.raises(B.OqError) as e:
+        B.oq_rq_plan(rot, B.oq_build_codebook(2048, 4))
+    assert e.value.code == 1
+    with pytest.raises(B.OqError) as e:
+        B.oq_debug_select_rq_kernel(7)
+    assert e.value.code == 1
+    # a width that is not a multiple of 128 has no fast path at all
+    with pytest.raises(B.OqError) as e:
+        B.oq_rq_plan(B.oq_make_rpbh(192, 64, 0), B.oq_build_codebook(192, 4))
+    assert e.value.code == 2
