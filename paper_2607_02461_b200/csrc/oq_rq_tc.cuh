@@ -344,32 +344,40 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const float inv_sqrt_h = rsqrtf((float)BLK);
     constexpr float mma_h = BLK < H ? (float)BLK : (float)H;   // the tensor-core product multiplies squared norms by this
     const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kq * 32);
+    // Pass 1 of one tile (sequence number n, tile i of its group): the sum of squares of the thread's 32 columns,
+    // zero for an unused row.
+    auto tile_sumsq = [&](uint32_t n, int i) {
+      const uint32_t slot = n % 3u;
+      warp_wait(acc_ready0 + 8 * slot, (n / 3u) & 1u, WAIT_ACC);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      uint32_t v[32];
+      tmem_load32(tmem_thr + slot * 128u, v);
+      unsigned long long qa = 0ull, qb = 0ull;      // two chains, fixed order
+#pragma unroll
+      for (int e = 0; e < 16; e += 2) {
+        const unsigned long long xa = pack2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
+        const unsigned long long xb = pack2(__uint_as_float(v[2 * e + 2]), __uint_as_float(v[2 * e + 3]));
+        qa = fma2(xa, xa, qa);
+        qb = fma2(xb, xb, qb);
+      }
+      float a0, a1, b0, b1;
+      unpack2(qa, a0, a1);
+      unpack2(qb, b0, b1);
+      return tile_valid(i, r) ? (a0 + a1) + (b0 + b1) : 0.f;
+    };
     uint32_t n0 = 0;                                  // sequence number of the group's first tile
     int it = 0;
-    for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it, n0 += (uint32_t)p.ntiles) {
-      const int row0 = grp * T;
-      // ---------------- pass 1: sums of squares of the rotated values, per half ----------------
-      float ssq0 = 0.f, ssq1 = 0.f;
+    // pass 1 of the CTA's first group; pass 1 of every later group is spread over the pass 2 of the group before it
+    float ssq0 = 0.f, ssq1 = 0.f;
+    if ((int)blockIdx.x < p.groups) {
       for (int i = 0; i < p.ntiles; ++i) {
-        const uint32_t n = n0 + (uint32_t)i, slot = n % 3u;
-        warp_wait(acc_ready0 + 8 * slot, (n / 3u) & 1u, WAIT_ACC);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t v[32];
-        tmem_load32(tmem_thr + slot * 128u, v);
-        unsigned long long qa = 0ull, qb = 0ull;      // two chains, fixed order
-#pragma unroll
-        for (int e = 0; e < 16; e += 2) {
-          const unsigned long long xa = pack2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-          const unsigned long long xb = pack2(__uint_as_float(v[2 * e + 2]), __uint_as_float(v[2 * e + 3]));
-          qa = fma2(xa, xa, qa);
-          qb = fma2(xb, xb, qb);
-        }
-        float a0, a1, b0, b1;
-        unpack2(qa, a0, a1);
-        unpack2(qb, b0, b1);
-        const float a = tile_valid(i, r) ? (a0 + a1) + (b0 + b1) : 0.f;
+        const float a = tile_sumsq((uint32_t)i, i);
         if (tile_half(i, q)) ssq1 += a; else ssq0 += a;
       }
+    }
+    for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it, n0 += (uint32_t)p.ntiles) {
+      const int row0 = grp * T;
+      const bool has_next = grp + stride < p.groups;
       // lanes of the warp that hold the same token add up (they differ in the lane bits above log2 th) ...
 #pragma unroll
       for (int o = 16; o >= 1; o >>= 1)
@@ -400,7 +408,9 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
       // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
       const float kappa0 = 1.0f / (sqrtf((float)BLK) * (s0 + 1e-10f) * p.poly.clamp);
       const float kappa1 = 1.0f / (sqrtf((float)BLK) * (s1 + 1e-10f) * p.poly.clamp);
-      // ---------------- pass 2: level search and packing ----------------
+      // ---------------- pass 2: level search and packing; pass 1 of the next group, one tile at a time ----------------
+      ssq0 = 0.f;
+      ssq1 = 0.f;
       for (int i = 0; i < p.ntiles; ++i) {
         const uint32_t n = n0 + (uint32_t)i, slot = n % 3u;
         const int half = tile_half(i, q), j = tile_block(i, r);
@@ -439,6 +449,12 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
 #pragma unroll
             for (int c = 0; c < BITS; ++c) dst[c] = words[c];
           }
+        }
+        // the next group's tile i went into the accumulator that this tile's pass 2 freed (3-tile groups) or one
+        // freed earlier: its MMAs ran while this warp packed
+        if (has_next) {
+          const float a = tile_sumsq(n + (uint32_t)p.ntiles, i);
+          if (tile_half(i, q)) ssq1 += a; else ssq0 += a;
         }
       }
     }
