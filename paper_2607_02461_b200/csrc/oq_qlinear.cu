@@ -306,6 +306,11 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
   cluster_sync_all();     // barriers of both CTAs are initialised before anyone arrives remotely
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
+  // Programmatic dependent launch: the set-up above may have run while the previous kernel of the stream (normally
+  // the rotate+quantize pass that produces Aq) was finishing; nothing below may start before that grid is complete.
+  // The next kernel may in turn be scheduled on SMs as this grid frees them.  (Both are no-ops in an ordinary launch.)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int kblocks = dim / PBK;
   const int tiles_n = (n_tokens + 255) / 256;
@@ -450,8 +455,7 @@ cudaError_t launch_pair(int sms, cudaStream_t st, const uint32_t* Aq, const floa
   int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev] : sms / 2;
   if (pairs > sms / 2) pairs = sms / 2;
   if (pairs > ntiles) pairs = ntiles;
-  k<<<2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st>>>(Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
-  return cudaGetLastError();
+  return launch_dependent(k, 2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
 }
 
 template <int BA, int BW>

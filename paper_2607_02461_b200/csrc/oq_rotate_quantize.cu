@@ -228,8 +228,7 @@ static cudaError_t launch_tc_bits(int tab, int grid, size_t smem, cudaStream_t s
   auto k = tab == 1 ? rq_tc_kernel<BITS, 1, BLK> : tab == 2 ? rq_tc_kernel<BITS, 2, BLK> : rq_tc_kernel<BITS, 0, BLK>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k<<<grid, rqtc::THREADS, smem, st>>>(prm);
-  return cudaGetLastError();
+  return launch_dependent(k, grid, rqtc::THREADS, smem, st, prm);
 }
 template <int BITS>
 static cudaError_t launch_tc_block(int block, int tab, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {

@@ -151,6 +151,10 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     for (int i = 0; i < 6; ++i) s_cnt[i] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // With programmatic dependent launch this CTA may have started while the previous kernel of the stream was still
+    // running: its results (the rows read here, buffers this kernel overwrites) are safe to touch only after this wait.
+    // Every other access to them in this CTA is ordered after it through barriers.  (A no-op in an ordinary launch.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // the first rows travel while the CTA builds its tables
     if ((int)blockIdx.x < p.groups)
       for (uint32_t hs = 0; hs < (uint32_t)ROWBUFS; ++hs) request_half(hs);
@@ -200,6 +204,9 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
+  // the next kernel of the stream may be scheduled on SMs as they become free (it waits for this grid to finish
+  // before it touches anything this grid reads or writes)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   auto warp_wait = [&](uint32_t bar, uint32_t parity, int code) {
     if (lane == 0) mbar_wait(bar, parity, abort_flag, p.status, code);
