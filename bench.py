@@ -325,6 +325,22 @@ def run_ours(args):
         if world > 1:
             dist.destroy_process_group()
         return
+    # Context line (a measurement of the box, not a dependency of the path): the library bf16 GEMM of the same
+    # shapes on dense operands, timed the same way.
+    mm_ms = []
+    for l in L:
+        Wd = torch.randn((l["m"], l["d"]), device=dev, dtype=torch.float32).mul_(0.02).to(torch.bfloat16)
+        for _ in range(2):
+            torch.matmul(l["X"], Wd.t(), out=l["Y"])
+        ts = []
+        for _ in range(5):
+            flush.zero_()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(); torch.matmul(l["X"], Wd.t(), out=l["Y"]); b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        mm_ms.append(sorted(ts)[len(ts) // 2])
+        del Wd
     pk = peaks()
     gemm_tf = sum(2 * tokens * l["m"] * l["d"] for l in L) / (float(np.sum(gemm_ms)) * 1e-3) / 1e12
     rq_b = sum(rq_bytes(tokens, l["d"], ba) for l in L)
@@ -359,6 +375,10 @@ def run_ours(args):
                                                        for i, l in enumerate(L)}},
         "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "context_torch_matmul_bf16": {"unit": "TFLOP/s", "note": "library GEMM on dense bf16 operands of the same shapes",
+                                      "all_layers": sum(2 * tokens * l["m"] * l["d"] for l in L) / (sum(mm_ms) * 1e-3) / 1e12,
+                                      "per_layer": {l["name"]: 2 * tokens * l["m"] * l["d"] / (mm_ms[i] * 1e-3) / 1e12
+                                                    for i, l in enumerate(L)}},
         "gpu_launches": 2 * len(L) * args.steps,
         "clocks": clocks, "device_status": status, "wall_s_timed_region": t_wall,
     }
