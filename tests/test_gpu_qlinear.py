@@ -133,3 +133,40 @@ def test_bounded_wait_gives_up_and_reports():
     wq, wr = B.oq_quantize_weights(_dev(synth.weights(16, d, 2)), rot, cb)
     y = B.oq_qlinear(xq, xs, cb, wq, wr, cb, d)
     assert torch.isfinite(y.float()).all() and B.oq_device_status() == 0
+
+
+def test_back_to_back_launches_into_shared_buffers_match_serialised_runs():
+    """Both kernels are launched with programmatic stream serialisation (a kernel may start while the previous one of
+    the stream is still running and waits inside before touching its data).  Layers launched back to back that reuse
+    ONE set of packed-activation buffers (every rotate+quantize overwrites what the GEMM before it reads) must give
+    bit-identical results to the same sequence with a device synchronisation after every kernel."""
+    import torch
+    d, m, n = 3072, 2048, 1000
+    rot, cb = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, 4)
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    Xs = [torch.randn((n, d), device="cuda", generator=gen).to(torch.bfloat16) * (k + 1) for k in range(4)]
+    W = (torch.randn((m, d), device="cuda", generator=gen) * 0.02).to(torch.bfloat16)
+    wq, wr = B.oq_quantize_weights(W, rot, cb)
+    xq = torch.empty((n, B.oq_packed_bytes(n, d, 4)[1]), dtype=torch.uint8, device="cuda")
+    xs = torch.empty(n, dtype=torch.float32, device="cuda")
+
+    def run(sync):
+        outs = []
+        for rep in range(3):
+            for X in Xs:
+                Y = torch.empty((n, m), dtype=torch.bfloat16, device="cuda")
+                B.oq_rotate_quantize_act(X, rot, cb, out_idx=xq, out_norm=xs)
+                if sync:
+                    torch.cuda.synchronize()
+                B.oq_qlinear(xq, xs, cb, wq, wr, cb, d, out=Y)
+                if sync:
+                    torch.cuda.synchronize()
+                outs.append(Y)
+        torch.cuda.synchronize()
+        return outs
+
+    ref = run(True)
+    got = run(False)
+    assert B.oq_device_status() == 0
+    for a, b in zip(ref, got):
+        assert torch.equal(a, b)
