@@ -195,8 +195,8 @@ int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows
 
 /* Test helper: selects the kernel behind oq_rotate_quantize_act / oq_quantize_weights for the following calls of
  * this process: 0 = choose by shape (default), 1 = general kernel (any block size; butterflies in shared memory),
- * 2 = register-butterfly kernel (blocks of 64, 128, 256), 3 = tensor-core kernel (blocks of 64, 128, 256; the block
- * Hadamard transform of Eq. 7 as a product with a 128 x 128 matrix of +-1).  A selected kernel that does not
+ * 2 = register-butterfly kernel (blocks of 64, 128, 256), 3 = tensor-core kernel (blocks of 64 to 4096; the block
+ * Hadamard transform of Eq. 7 as a product with a 128 x 128 matrix of +-1, plus butterfly stages for larger blocks).  A selected kernel that does not
  * support the shape falls back to the general one.  All three compute the same function; the parity tests run
  * each of them.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
 int oq_debug_select_rq_kernel(int which);

@@ -193,15 +193,20 @@ static int g_forced_kernel = 0;
 // shared memory beside the Hadamard tile.
 struct TcPlan {
   int ths, pairs, ntiles;
+  int stages;       // blocks of 512 and more: log2(block / 128) butterfly stages after the tensor-core product
   int tab;          // 0: tables in global memory, 1: both in shared memory, 2: 16-bit offsets in shared memory
   size_t smem;
   double fill;      // used rows of the operand tiles / all rows
 };
 static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
-  if ((block != 64 && block != 128 && block != 256) || !cb->poly.ok) return false;
+  if (block < 64 || block > 4096 || (block & (block - 1)) || !cb->poly.ok) return false;
   const size_t kMaxSmem = 227 * 1024;
   const int kblocks = dim / 128;
-  for (int ths = 3; ths >= 0; --ths) {
+  // the 2^stages sub-blocks of th tokens must sit in one warp's 32 tile rows
+  int stages = 0;
+  while ((128 << stages) < block) ++stages;
+  plan->stages = stages;
+  for (int ths = stages > 2 ? 5 - stages : 3; ths >= 0; --ths) {
     const int th = 1 << ths;
     const int pairs = th * kblocks;
     if (pairs > rqtc::MAX_PAIRS) continue;
@@ -234,6 +239,7 @@ template <int BITS>
 static cudaError_t launch_tc_block(int block, int tab, int grid, size_t smem, cudaStream_t st, const RqTcParams& prm) {
   if (block == 64) return launch_tc_bits<BITS, 64>(tab, grid, smem, st, prm);
   if (block == 256) return launch_tc_bits<BITS, 256>(tab, grid, smem, st, prm);
+  if (block > 256) return launch_tc_bits<BITS, 512>(tab, grid, smem, st, prm);
   return launch_tc_bits<BITS, 128>(tab, grid, smem, st, prm);
 }
 
@@ -266,6 +272,7 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
     prm.groups = (rows + T - 1) / T;
     prm.ths = tp.ths; prm.pairs = tp.pairs; prm.ntiles = tp.ntiles;
     prm.bf16_norm = kBf16Norm ? 1 : 0;
+    prm.stages = tp.stages;
     prm.status = status;
     int grid = sms < prm.groups ? sms : prm.groups;
     if (cb->bits == 4) e = launch_tc_block<4>(rot->block, tp.tab, grid, tp.smem, st, prm);

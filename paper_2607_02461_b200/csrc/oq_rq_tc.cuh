@@ -1,4 +1,4 @@
-// Fused rotate+quantize kernel for Hadamard blocks of 64, 128 and 256 with the block transform on the tensor cores.
+// Fused rotate+quantize kernel for Hadamard blocks of 64 to 4096 with the block transform on the tensor cores.
 //
 // The rotation of Eq. 7 / Eq. 4 is  z = blkdiag(H_128 D_j) P x : a gather, a sign flip and, per block of 128
 // rotated coordinates, a product with the 128 x 128 matrix of +-1.  Butterflies in registers cost ~6
@@ -7,7 +7,9 @@
 // (token, block) pairs by H_128 (entries +-1 are exact in bf16, the inputs are bf16 already, the sums are
 // accumulated in fp32 in tensor memory).  The rest of the path reads tensor memory twice: once for the row
 // norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.  Blocks of 64 use a block-diagonal
-// operand (two blocks per 128 coordinates); blocks of 256 add one butterfly stage across two tile rows.
+// operand (two blocks per 128 coordinates); a block of 128 * 2^S coordinates (S = 1 .. 5) is H_{2^S} (x) H_128 in
+// natural order, so after the tensor-core product its 2^S sub-blocks, which sit th tile rows apart in one warp,
+// go through S butterfly stages of one shuffle and one FMA per coordinate.
 //
 // Work units.  A group is 2 th consecutive rows (th = 1, 2, 4 or 8 tokens per HALF group, chosen so that the
 // P = th * dim / 128 (token, block) pairs of a half number at most 192).  Each half has its own row buffer and
@@ -57,6 +59,7 @@ struct RqTcParams {
   int pairs;                // P = th * dim / 128 pairs per half (<= 192)
   int ntiles;               // 2 (P <= 128) or 3
   int bf16_norm;            // 1: norms stored as bf16 (weights), 0: fp32 (activations)
+  int stages;               // BLK = 512 only: the Hadamard block is 128 << stages (2 .. 5), th << stages <= 32
   int* status;
 };
 
@@ -84,7 +87,8 @@ __host__ __device__ constexpr uint32_t row_pitch_bytes(int dim) { return 2u * (u
 
 // TAB: where the gather tables live.  0: global memory (read-only path); 1: both copied to shared memory (32-bit
 // offsets, masks); 2: offsets copied to shared memory as 16-bit values, masks stay in global memory.
-// BLK: the Hadamard block, 64, 128 or 256 (256: one butterfly stage across two tile rows after the tensor-core product).
+// BLK: the Hadamard block, 64, 128 or 256 (256: one butterfly stage across two tile rows after the tensor-core product);
+// 512 stands for every larger block, 128 << p.stages, with p.stages butterfly stages.
 template <int BITS, int TAB, int BLK>
 __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParams p) {
   using namespace rqtc;
@@ -348,7 +352,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const int r = q * 32 + lane;                     // row of the tile = tensor-memory lane
     const int tl = lane & (th - 1);
     const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
-    const float inv_sqrt_h = rsqrtf((float)BLK);
+    const float blk_f = BLK == 512 ? (float)(H << p.stages) : (float)BLK;      // coordinates per Hadamard block
+    const float inv_sqrt_h = rsqrtf(blk_f);
     constexpr float mma_h = BLK < H ? (float)BLK : (float)H;   // the tensor-core product multiplies squared norms by this
     const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(kq * 32);
     // Pass 1 of one tile (sequence number n, tile i of its group): the sum of squares of the thread's 32 columns,
@@ -413,8 +418,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
       }
       const float s0 = __shfl_sync(0xffffffffu, nrm, tl), s1 = __shfl_sync(0xffffffffu, nrm, 8 + tl);
       // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
-      const float kappa0 = 1.0f / (sqrtf((float)BLK) * (s0 + 1e-10f) * p.poly.clamp);
-      const float kappa1 = 1.0f / (sqrtf((float)BLK) * (s1 + 1e-10f) * p.poly.clamp);
+      const float kappa0 = 1.0f / (sqrtf(blk_f) * (s0 + 1e-10f) * p.poly.clamp);
+      const float kappa1 = 1.0f / (sqrtf(blk_f) * (s1 + 1e-10f) * p.poly.clamp);
       // ---------------- pass 2: level search and packing; pass 1 of the next group, one tile at a time ----------------
       ssq0 = 0.f;
       ssq1 = 0.f;
@@ -435,6 +440,19 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
             const float mine = __uint_as_float(vb[e]);
             const float other = __shfl_xor_sync(0xffffffffu, mine, th);
             vb[e] = __float_as_uint(fmaf(mine, sg, other));      // low half: mine + other; high half: other - mine
+          }
+        } else if constexpr (BLK == 512) {
+          // H_{2^S} (x) H_128: sub-block u of a block sits in lane bit positions log2(th) .. log2(th) + S - 1; stage s
+          // combines the rows that differ in bit s of u (sum in the row with the bit clear, difference in the other)
+          for (int s = 0; s < p.stages; ++s) {
+            const int bit = th << s;
+            const float sg = (lane & bit) ? -1.f : 1.f;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float mine = __uint_as_float(vb[e]);
+              const float other = __shfl_xor_sync(0xffffffffu, mine, bit);
+              vb[e] = __float_as_uint(fmaf(mine, sg, other));
+            }
           }
         }
         const int row = row0 + half * th + tl;

@@ -102,6 +102,43 @@ def test_tensor_core_kernel_on_blocks_of_64_and_256(d, n, block, bits):
     assert check_rows(xb, block, 5, bits, kernel=TENSOR) <= 1e-4
 
 
+@pytest.mark.parametrize("bits", [4, 3, 2])
+@pytest.mark.parametrize("d,block,n", [(3072, 1024, 67), (3072, 512, 67), (5120, 1024, 35), (5120, 512, 35),
+                                       (12288, 4096, 21), (12288, 2048, 21), (12288, 1024, 21), (13824, 512, 9),
+                                       (1024, 1024, 40), (2048, 2048, 19), (4096, 4096, 9), (1024, 512, 67)])
+def test_tensor_core_kernel_on_blocks_of_512_to_4096(d, block, n, bits):
+    """The paper's default block is the largest power of two that divides the width (1024 for 3072 and 5120, 4096 for
+    12288, 512 for 13824): H_{2^S} (x) H_128, i.e. S butterfly stages across the tile rows of a block after the
+    tensor-core product.  The oracle applies the full-size Hadamard matrix."""
+    xb = synth.activations(n, d, seed=1500 + bits)
+    rot, cb = B.oq_make_rpbh(d, block, 6), B.oq_build_codebook(d, bits)
+    B.oq_debug_select_rq_kernel(TENSOR)
+    assert B.oq_rq_plan(rot, cb)[0] == TENSOR
+    assert check_rows(xb, block, 6, bits, kernel=TENSOR) <= 1e-4
+
+
+@pytest.mark.parametrize("n", [1, 3, 8, 9, 17])
+@pytest.mark.parametrize("d,block", [(3072, 1024), (12288, 4096), (13824, 512)])
+def test_large_blocks_with_few_rows_match_the_general_kernel(n, d, block):
+    """Ragged groups with the multi-stage butterflies: rows that do not exist share warps with rows that do."""
+    import torch
+    xb = synth.activations(n, d, seed=1600 + n)
+    rot, cb = B.oq_make_rpbh(d, block, 4), B.oq_build_codebook(d, 4)
+    X = _dev(xb)
+    B.oq_debug_select_rq_kernel(GENERAL)
+    ref_idx, ref_norm = B.oq_rotate_quantize_act(X, rot, cb)
+    B.oq_debug_select_rq_kernel(AUTO)
+    assert B.oq_rq_plan(rot, cb)[0] == TENSOR
+    idx, norm = B.oq_rotate_quantize_act(X, rot, cb)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.allclose(norm, ref_norm, rtol=2e-6, atol=0)
+    a = B.oq_unpack_indices(idx, n, d, 4).to(torch.int16)
+    b = B.oq_unpack_indices(ref_idx, n, d, 4).to(torch.int16)
+    diff = (a - b).abs()
+    assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 2e-4
+
+
 @pytest.mark.parametrize("kernel", [REGISTERS, TENSOR])
 def test_kernels_agree_with_each_other_on_many_groups(kernel):
     """More row groups than CTAs (several pipeline rounds per CTA), ragged last group: same packed words and

@@ -132,7 +132,11 @@ def test_level_search_polynomial_counts_boundaries(dim, bits):
     (3072, 64, 3, 16, 3),       # blocks of 64 and 256 use the same 128-coordinate tile rows
     (3072, 256, 3, 16, 3),
     (1024, 256, 2, 8, 0),
-    (3072, 1024, 1, 1, 0),      # the paper's default block for this width: general kernel
+    (3072, 1024, 3, 8, 2),      # the paper's default blocks: the 2^S sub-blocks of a token must share a warp's
+    (5120, 1024, 3, 8, 3),      # 32 tile rows, so at most 32 / 2^S tokens per half group
+    (12288, 4096, 3, 2, 2),
+    (13824, 512, 3, 2, 2),
+    (1024, 1024, 1, 1, 0),      # a quarter-full tile: general kernel
 ])
 def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
     """Host-side launch planning (no device needed): kernel choice and group shape for the benchmark widths."""
