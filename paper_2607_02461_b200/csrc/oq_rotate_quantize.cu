@@ -202,11 +202,11 @@ static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
   if (block < 64 || block > 4096 || (block & (block - 1)) || !cb->poly.ok) return false;
   const size_t kMaxSmem = 227 * 1024;
   const int kblocks = dim / 128;
-  // the 2^stages sub-blocks of th tokens must sit in one warp's 32 tile rows
+  // blocks above 256: a row's token must be the same in every tile of a group, i.e. th * 2^stages divides 64
   int stages = 0;
   while ((128 << stages) < block) ++stages;
   plan->stages = stages;
-  for (int ths = stages > 2 ? 5 - stages : 3; ths >= 0; --ths) {
+  for (int ths = stages > 3 ? 6 - stages : 3; ths >= 0; --ths) {
     const int th = 1 << ths;
     const int pairs = th * kblocks;
     if (pairs > rqtc::MAX_PAIRS) continue;

@@ -8,8 +8,8 @@
 // accumulated in fp32 in tensor memory).  The rest of the path reads tensor memory twice: once for the row
 // norms (||H x'||^2 = 128 ||x||^2), once for the level search and packing.  Blocks of 64 use a block-diagonal
 // operand (two blocks per 128 coordinates); a block of 128 * 2^S coordinates (S = 1 .. 5) is H_{2^S} (x) H_128 in
-// natural order, so after the tensor-core product its 2^S sub-blocks, which sit th tile rows apart in one warp,
-// go through S butterfly stages of one shuffle and one FMA per coordinate.
+// natural order, so after the tensor-core product its 2^S sub-blocks, which sit in adjacent tile rows of one
+// warp, go through S butterfly stages of one shuffle and one FMA per coordinate.
 //
 // Work units.  A group is 2 th consecutive rows (th = 1, 2, 4 or 8 tokens per HALF group, chosen so that the
 // P = th * dim / 128 (token, block) pairs of a half number at most 192).  Each half has its own row buffer and
@@ -59,7 +59,7 @@ struct RqTcParams {
   int pairs;                // P = th * dim / 128 pairs per half (<= 192)
   int ntiles;               // 2 (P <= 128) or 3
   int bf16_norm;            // 1: norms stored as bf16 (weights), 0: fp32 (activations)
-  int stages;               // BLK = 512 only: the Hadamard block is 128 << stages (2 .. 5), th << stages <= 32
+  int stages;               // BLK = 512 only: the Hadamard block is 128 << stages (2 .. 5), th << stages <= 64
   int* status;
 };
 
@@ -216,10 +216,19 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     if (lane == 0) mbar_wait(bar, parity, abort_flag, p.status, code);
     __syncwarp();
   };
-  // Which pair row r of tile i holds: its half, its block, and whether the row is in use.  (q = r / 32.)
+  // Which pair row r of tile i holds: its half, its block of 128 coordinates, and whether the row is in use.
+  // (q = r / 32.)  Pair number = block * th + token; for blocks above 256 the S low bits of the block number move
+  // below the token bits, (block_hi * th + token) * 2^S + block_lo, so that the sub-blocks of one Hadamard block are
+  // adjacent rows.  The token of a row is the same in every tile (th * 2^S divides 64).
+  const int lg_lo = BLK == 512 ? p.stages : 0;
   auto tile_half = [&](int i, int q) { return nt3 ? (i == 0 ? 0 : (i == 2 ? 1 : (q >> 1))) : i; };
-  auto tile_block = [&](int i, int r) { return ((nt3 && i == 1) ? 128 + (r & 63) : r) >> p.ths; };
+  auto tile_block = [&](int i, int r) {
+    const int pr = (nt3 && i == 1) ? 128 + (r & 63) : r;
+    if constexpr (BLK == 512) return ((pr >> (lg_lo + p.ths)) << lg_lo) | (pr & ((1 << lg_lo) - 1));
+    else return pr >> p.ths;
+  };
   auto tile_valid = [&](int i, int r) { return nt3 ? (i != 1 || (r & 63) < rem) : r < p.pairs; };
+  auto row_token = [&](int r) { return ((r & 63) >> lg_lo) & (th - 1); };
 
   if (warp == MMA_WARP) {
     // ------------------------------- MMA issuer -------------------------------
@@ -253,7 +262,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const int gw = warp - COMPUTE_WARPS;
     const int gq = gw & 3, kh = gw >> 2;              // lane quarter of the tile, half of the 128 coordinates
     const int r = gq * 32 + lane;                     // row of the operand tile
-    const int tl = lane & (th - 1);                   // token within its half (the same in every tile)
+    const int tl = row_token(r);                      // token within its half (the same in every tile)
     const uint32_t a_thr = tmem + ((uint32_t)(gq * 32) << 16) + A_COL0 + (uint32_t)kh * 32u;   // + 64 * buffer
     uint32_t n = 0;
     int it = 0;
@@ -350,7 +359,9 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     // ------------------------------- compute warps -------------------------------
     const int q = warp & 3, kq = warp >> 2;          // tensor-memory lane quarter, column quarter
     const int r = q * 32 + lane;                     // row of the tile = tensor-memory lane
-    const int tl = lane & (th - 1);
+    const int tl = row_token(r);
+    // lane bits that number the token (the other bits run over the blocks of that token)
+    const int tok_bits = BLK == 512 ? (((th - 1) << lg_lo) & 31) : th - 1;
     const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
     const float blk_f = BLK == 512 ? (float)(H << p.stages) : (float)BLK;      // coordinates per Hadamard block
     const float inv_sqrt_h = rsqrtf(blk_f);
@@ -390,17 +401,18 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     for (int grp = blockIdx.x; grp < p.groups; grp += stride, ++it, n0 += (uint32_t)p.ntiles) {
       const int row0 = grp * T;
       const bool has_next = grp + stride < p.groups;
-      // lanes of the warp that hold the same token add up (they differ in the lane bits above log2 th) ...
+      // lanes of the warp that hold the same token add up (they differ in the lane bits that are not token bits) ...
 #pragma unroll
       for (int o = 16; o >= 1; o >>= 1)
-        if (o >= th) {
+        if (BLK == 512 ? !(o & tok_bits) : o >= th) {
           ssq0 += __shfl_xor_sync(0xffffffffu, ssq0, o);
           ssq1 += __shfl_xor_sync(0xffffffffu, ssq1, o);
         }
+      // (with large blocks a warp may hold only some of the tokens; the slots of the others stay zero)
       float* part = s_part + (it & 1) * (COMPUTE_WARPS * 16);
-      if (lane < th) {
-        part[warp * 16 + lane] = ssq0;
-        part[warp * 16 + 8 + lane] = ssq1;
+      if ((lane & ~tok_bits) == 0) {
+        part[warp * 16 + tl] = ssq0;
+        part[warp * 16 + 8 + tl] = ssq1;
       }
       asm volatile("bar.sync 1, %0;" ::"n"(COMPUTE_THREADS) : "memory");
       // ... and the 16 warps' partial sums in a fixed order: lane L adds 8 warps for slot L & 15
@@ -442,10 +454,10 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
             vb[e] = __float_as_uint(fmaf(mine, sg, other));      // low half: mine + other; high half: other - mine
           }
         } else if constexpr (BLK == 512) {
-          // H_{2^S} (x) H_128: sub-block u of a block sits in lane bit positions log2(th) .. log2(th) + S - 1; stage s
-          // combines the rows that differ in bit s of u (sum in the row with the bit clear, difference in the other)
+          // H_{2^S} (x) H_128: sub-block u of a block is the low S bits of the lane; stage s combines the rows that
+          // differ in bit s of u (sum in the row with the bit clear, difference in the other)
           for (int s = 0; s < p.stages; ++s) {
-            const int bit = th << s;
+            const int bit = 1 << s;
             const float sg = (lane & bit) ? -1.f : 1.f;
 #pragma unroll
             for (int e = 0; e < 32; ++e) {

@@ -132,9 +132,9 @@ def test_level_search_polynomial_counts_boundaries(dim, bits):
     (3072, 64, 3, 16, 3),       # blocks of 64 and 256 use the same 128-coordinate tile rows
     (3072, 256, 3, 16, 3),
     (1024, 256, 2, 8, 0),
-    (3072, 1024, 3, 8, 2),      # the paper's default blocks: the 2^S sub-blocks of a token must share a warp's
-    (5120, 1024, 3, 8, 3),      # 32 tile rows, so at most 32 / 2^S tokens per half group
-    (12288, 4096, 3, 2, 2),
+    (3072, 1024, 3, 16, 3),     # the paper's default blocks: same group shapes as blocks of 128
+    (5120, 1024, 3, 8, 3),
+    (12288, 4096, 3, 4, 3),
     (13824, 512, 3, 2, 2),
     (1024, 1024, 1, 1, 0),      # a quarter-full tile: general kernel
 ])
