@@ -13,6 +13,7 @@ rpbh      randomized permuted block-Hadamard rotation (Eq. 9), dense definition
 codebook  Lloyd-Max scalar codebook for the sphere-coordinate marginal (Eq. 2-3)
 quantize  per-row rotate -> norm -> nearest centroid (Eq. 4-8, Algorithm 1)
 qlinear   product of the decoded operands with both norms re-attached
+adaln     AdaLN modulation projection: weight-only INT4 round-to-nearest in groups of 64, bf16 activations
 
 Parity pins: every function here is pinned by tests/test_oracle_*.py against
 closed forms, exact invariants, brute force and classical published tables.
