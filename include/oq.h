@@ -178,6 +178,35 @@ int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out
  * OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
 int oq_device_status(int* status);
 
+/* ---- AdaLN modulation projections (weight-only INT4, bf16 activations) ----------------------------- */
+
+/* The AdaLN modulation projections are not rotated: their weights are quantized to INT4 by round-to-nearest in
+ * groups of 64 input coordinates and their input, one conditioning token per sample, stays in bf16 (the
+ * supplementary section on quantized layers; Sec. 5.1).  The grid, on which the paper is silent, is symmetric:
+ * scale = bf16(max |w| / 7) per (row, group), q = clamp(rint(w / scale), -8, 7), q = 0 where the scale is 0
+ * (divisions in fp32).  Bytes of the two device buffers for an m x dim weight: *wq_bytes = m * dim / 2,
+ * *scale_bytes = 2 * m * dim / 64.  m must be a multiple of 16, dim of 64 (OQ_ERR_UNSUPPORTED otherwise). */
+int oq_adaln_packed_bytes(int m, int dim, size_t* wq_bytes, size_t* scale_bytes);
+
+/* Offline, on the GPU: W_bf16 (device, row-major [m][ldw], ldw >= dim, ldw % 8 == 0, 16-byte aligned) ->
+ * Wq (device, wq_bytes, 16-byte aligned; layout private to the library: the order in which the tensor-core
+ * fragments of oq_adaln_linear consume the nibbles) and scales (device, scale_bytes, 16-byte aligned).
+ * Asynchronous on `stream`.  Errors: OQ_ERR_INVALID_ARG, OQ_ERR_UNSUPPORTED, OQ_ERR_ALIGNMENT, OQ_ERR_CUDA. */
+int oq_adaln_quantize_weights(const void* W_bf16, int m, int dim, int ldw, void* Wq, void* scales, void* stream);
+
+/* Y[n][row] = sum over groups of scale * sum_i q_i * X[n][i]  (products of a group accumulated in fp32 on the
+ * tensor cores, groups added in fp32 in a fixed order: results are bit-reproducible).  X_bf16: device,
+ * [n_tokens][ldx], ldx >= dim, ldx % 8 == 0, 16-byte aligned.  Y: device, [n_tokens][ldy], ldy >= m, OQ_BF16 or
+ * OQ_F32.  One pass over the weights per 8 tokens (the layer sees one token per sample).  The tokens of a pass are
+ * staged in shared memory: min(n_tokens, 8) * (2 * dim + 16) bytes + 8 KB must fit in 227 KB (dim <= 13952 for 8).
+ * Asynchronous on `stream`; nothing is allocated.  Errors as above. */
+int oq_adaln_linear(const void* X_bf16, int n_tokens, int ldx, const void* Wq, const void* scales, int m, int dim,
+                    void* Y, int ldy, int y_dtype, void* stream);
+
+/* Test helper: logical values of the private layout.  q_int8: device int8 [m][dim] (-8..7); scale_bf16: device
+ * bf16 bit patterns [m][dim / 64]. */
+int oq_adaln_unpack(const void* Wq, const void* scales, int m, int dim, void* q_int8, void* scale_bf16, void* stream);
+
 /* Self-test of the bounded device-side waits the GEMM pipeline is built on: launches one thread that waits
  * about a millisecond on a barrier nobody arrives at.  The wait gives up by itself (the kernel ends
  * normally, nothing hangs or traps) and records code 9; the following oq_device_status() must return

@@ -51,6 +51,10 @@ def lib():
             "oq_selftest_bounded_wait": (i, [vp]),
             "oq_debug_select_rq_kernel": (i, [i]),
             "oq_rq_plan": (i, [vp, vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(sz)]),
+            "oq_adaln_packed_bytes": (i, [i, i, C.POINTER(sz), C.POINTER(sz)]),
+            "oq_adaln_quantize_weights": (i, [vp, i, i, i, vp, vp, vp]),
+            "oq_adaln_linear": (i, [vp, i, i, vp, vp, i, i, vp, i, i, vp]),
+            "oq_adaln_unpack": (i, [vp, vp, i, i, vp, vp, vp]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
         for name, (res, args) in sig.items():
@@ -227,6 +231,44 @@ def oq_rq_plan(rot, cb):
 
 def oq_debug_select_rq_kernel(which):
     _check(lib().oq_debug_select_rq_kernel(int(which)))
+
+
+def oq_adaln_packed_bytes(m, dim):
+    a, b = C.c_size_t(), C.c_size_t()
+    _check(lib().oq_adaln_packed_bytes(m, dim, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def oq_adaln_quantize_weights(W):
+    """W: CUDA bf16 [m, d].  Returns (packed nibbles uint8 [m * d / 2], scales uint8 [2 * m * d / 64])."""
+    import torch
+    m, d = W.shape
+    wq_bytes, sc_bytes = oq_adaln_packed_bytes(m, d)
+    Wq = torch.empty(wq_bytes, dtype=torch.uint8, device=W.device)
+    Sc = torch.empty(sc_bytes, dtype=torch.uint8, device=W.device)
+    _check(lib().oq_adaln_quantize_weights(_ptr(W), m, d, W.stride(0) if m > 1 else d, _ptr(Wq), _ptr(Sc), _stream()))
+    return Wq, Sc
+
+
+def oq_adaln_linear(X, Wq, Sc, m, out=None, out_dtype=None):
+    """X: CUDA bf16 [n, d].  Returns Y [n, m] (bf16 by default, fp32 when out_dtype is torch.float32)."""
+    import torch
+    n, d = X.shape
+    if out is None:
+        out = torch.empty((n, m), dtype=out_dtype or torch.bfloat16, device=X.device)
+    ydt = OQ_F32 if out.dtype == torch.float32 else OQ_BF16
+    _check(lib().oq_adaln_linear(_ptr(X), n, X.stride(0) if n > 1 else d, _ptr(Wq), _ptr(Sc), m, d, _ptr(out),
+                                 out.stride(0) if n > 1 else m, ydt, _stream()))
+    return out
+
+
+def oq_adaln_unpack(Wq, Sc, m, dim):
+    """Returns (q int8 [m, d], scale bf16 [m, d / 64]) on the device."""
+    import torch
+    q = torch.empty((m, dim), dtype=torch.int8, device=Wq.device)
+    s = torch.empty((m, dim // 64), dtype=torch.bfloat16, device=Wq.device)
+    _check(lib().oq_adaln_unpack(_ptr(Wq), _ptr(Sc), m, dim, _ptr(q), _ptr(s), _stream()))
+    return q, s
 
 
 def oq_version():

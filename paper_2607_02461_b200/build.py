@@ -9,7 +9,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liboq.so")
-SOURCES = ["oq_host.cu", "oq_rotate_quantize.cu", "oq_qlinear.cu", "oq_forward_host.cu", "oq_noalloc.cu"]
+SOURCES = ["oq_host.cu", "oq_rotate_quantize.cu", "oq_qlinear.cu", "oq_forward_host.cu", "oq_noalloc.cu",
+           "oq_adaln.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 

@@ -3,6 +3,7 @@
     python -m paper_2607_02461_b200.microbench rq   --tokens 17776 --dim 3072 --bits 4 --block 128
     python -m paper_2607_02461_b200.microbench gemm --tokens 4608 --dim 3072 --m 9216 --bits-a 4 --bits-w 4
     python -m paper_2607_02461_b200.microbench sweep [--quick]     # rotate+quantize bandwidth sweep
+    python -m paper_2607_02461_b200.microbench adaln --tokens 1 --dim 3072 --m 18432   # AdaLN INT4 projection
 
 Inputs are synthetic and generated on the GPU (normal values, per-token log-uniform scale, 1% of the
 channels multiplied by 30); these runs time the kernels, parity is covered by the tests.
@@ -67,9 +68,22 @@ def run_gemm(n, d, m, ba, bw, iters):
             "ms_min": best, "flops": fl, "tflops": fl / med / 1e9, "tflops_best": fl / best / 1e9}
 
 
+def run_adaln(n, d, m, iters):
+    W = (torch.randn((m, d), device="cuda") * 0.02).to(torch.bfloat16)
+    Wq, Sc = B.oq_adaln_quantize_weights(W)
+    del W
+    X = torch.nn.functional.silu(torch.randn((n, d), device="cuda")).to(torch.bfloat16)
+    Y = torch.empty((n, m), dtype=torch.bfloat16, device="cuda")
+    med, best = time_kernel(lambda: B.oq_adaln_linear(X, Wq, Sc, m, out=Y), iters)
+    passes = (n + 7) // 8
+    nbytes = passes * (m * d // 2 + 2 * m * d // 64) + 2 * n * d + 2 * n * m
+    return {"kernel": "adaln_linear", "tokens": n, "dim": d, "m": m, "ms_median": med, "ms_min": best, "bytes": nbytes,
+            "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("mode", choices=["rq", "gemm", "sweep"])
+    ap.add_argument("mode", choices=["rq", "gemm", "sweep", "adaln"])
     ap.add_argument("--tokens", type=int, default=17776)
     ap.add_argument("--dim", type=int, default=3072)
     ap.add_argument("--m", type=int, default=9216)
@@ -87,6 +101,8 @@ def main(argv=None):
         print(json.dumps(run_rq(a.tokens, a.dim, a.bits, a.block, a.iters)))
     elif a.mode == "gemm":
         print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters)))
+    elif a.mode == "adaln":
+        print(json.dumps(run_adaln(a.tokens, a.dim, a.m, a.iters)))
     else:
         toks = [4608, 32760] if a.quick else [4608, 17776, 32760, 75600]
         for n in toks:
