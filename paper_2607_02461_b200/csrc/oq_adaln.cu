@@ -29,7 +29,8 @@ constexpr int GROUP = 64;
 constexpr int WARPS = 8, THREADS = WARPS * 32;
 constexpr int RT = 2;              // row tiles (of 16 rows) per CTA
 constexpr int MAXN = 8;            // tokens per launch (the n of m16n8k16)
-constexpr int PF = 3;              // groups in flight per warp
+constexpr int PF = 2;              // groups in flight per warp
+constexpr int CTAS_PER_SM = 4;
 
 __device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
   uint32_t d;
@@ -37,34 +38,38 @@ __device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
   return d;
 }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+// d = a * b + c (c may be a literal zero: no register is spent on it)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1, float c0, float c1,
+                                               float c2, float c3) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
 }
 
-// Grid: one CTA per RT row tiles.  Warp w of the CTA takes the groups w, w + 8, ...; the eight partial results meet
-// in shared memory and are added in a fixed order (bit-reproducible output).
-__global__ void __launch_bounds__(THREADS) adaln_linear_kernel(const uint4* __restrict__ Wq, const uint32_t* __restrict__ S,
+// Grid: CTA b takes the row tiles [b * tiles_per_cta, (b + 1) * tiles_per_cta), RT at a time (one wave of CTAs for
+// the layer's real sizes: the activations are staged once per CTA).  Warp w of the CTA takes the groups w, w + 8,
+// ...; the eight partial results meet in shared memory and are added in a fixed order (bit-reproducible output).
+__global__ void __launch_bounds__(THREADS, CTAS_PER_SM) adaln_linear_kernel(const uint4* __restrict__ Wq, const uint32_t* __restrict__ S,
                                                                const __nv_bfloat16* __restrict__ X, int n, int ldx, int m,
-                                                               int dim, void* __restrict__ Y, int ldy, int f32_out) {
+                                                               int dim, int tiles_per_cta, void* __restrict__ Y, int ldy,
+                                                               int f32_out) {
   extern __shared__ uint4 smem_dyn4[];
-  uint32_t* xs = reinterpret_cast<uint32_t*>(smem_dyn4);      // [n][dim / 2 + 4] words: rows 4 banks apart
+  uint32_t* xs = reinterpret_cast<uint32_t*>(smem_dyn4);      // [n + 1][dim / 2 + 4] words: rows 4 banks apart; row n is zero
   const int pitch_w = dim / 2 + 4;
-  float* red = reinterpret_cast<float*>(xs + (size_t)n * pitch_w);   // [WARPS][RT * 16][8]
+  float* red = reinterpret_cast<float*>(xs + (size_t)(n + 1) * pitch_w);   // [WARPS][RT * 16][8]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, tig = lane & 3;
   const int G = dim / GROUP, tiles = m / 16;
-  const int tile0 = blockIdx.x * RT;
+  const int tile_end = min(tiles, ((int)blockIdx.x + 1) * tiles_per_cta);
+  int tile0 = blockIdx.x * tiles_per_cta;
 
   auto load_group = [&](int grp, uint4 (&w)[RT], uint32_t (&sc)[RT]) {
 #pragma unroll
     for (int t = 0; t < RT; ++t) {
-      if (grp < G && tile0 + t < tiles) {
-        const size_t tg = (size_t)(tile0 + t) * G + grp;
-        w[t] = __ldcs(Wq + tg * 32 + lane);
-        sc[t] = __ldg(S + tg * 8 + g);
+      if (grp < G && tile0 + t < tile_end) {
+        const uint32_t tg = (uint32_t)(tile0 + t) * (uint32_t)G + (uint32_t)grp;      // < 2^26: the host checks m * dim < 2^36
+        w[t] = __ldcs(Wq + (tg * 32u + (uint32_t)lane));
+        sc[t] = __ldg(S + (tg * 8u + (uint32_t)g));
       } else {
         w[t] = make_uint4(0u, 0u, 0u, 0u);
         sc[t] = 0u;                                  // a zero scale removes whatever the nibbles decode to
@@ -82,73 +87,85 @@ __global__ void __launch_bounds__(THREADS) adaln_linear_kernel(const uint4* __re
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(X + (size_t)row * ldx) + c);
     *reinterpret_cast<uint4*>(xs + (size_t)row * pitch_w + c * 4) = v;
   }
+  for (int i = tid; i < pitch_w / 4; i += THREADS) *reinterpret_cast<uint4*>(xs + (size_t)n * pitch_w + i * 4) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
+  // column g of the product is token g; the columns past the last token read the zero row
+  const uint32_t* xrow = xs + (g < n ? g : n) * pitch_w + tig;
 
-  float acc[RT][4];
+  for (; tile0 < tile_end; tile0 += RT) {
+    float acc[RT][4];
 #pragma unroll
-  for (int t = 0; t < RT; ++t)
+    for (int t = 0; t < RT; ++t)
 #pragma unroll
-    for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
-  const bool has_token = g < n;                       // column g of the product is token g
-  const uint32_t* xrow = xs + (size_t)(has_token ? g : 0) * pitch_w + tig;
-
-  for (int it = 0; warp + it * WARPS < G; it += PF) {
+      for (int e = 0; e < 4; ++e) acc[t][e] = 0.f;
+    for (int it = 0; warp + it * WARPS < G; it += PF) {
 #pragma unroll
-    for (int u = 0; u < PF; ++u) {
-      const int grp = warp + (it + u) * WARPS;
-      if (grp < G) {                                  // warp-uniform
-        uint4 w[RT];
-        uint32_t sc[RT];
+      for (int u = 0; u < PF; ++u) {
+        const int grp = warp + (it + u) * WARPS;
+        if (grp < G) {                                  // warp-uniform
+          uint4 w[RT];
+          uint32_t sc[RT];
 #pragma unroll
-        for (int t = 0; t < RT; ++t) {
-          w[t] = wbuf[u][t];
-          sc[t] = sbuf[u][t];
-        }
-        load_group(grp + PF * WARPS, wbuf[u], sbuf[u]);
-        uint32_t b[4][2];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          b[c][0] = has_token ? xrow[grp * 32 + c * 8] : 0u;
-          b[c][1] = has_token ? xrow[grp * 32 + c * 8 + 4] : 0u;
-        }
-#pragma unroll
-        for (int t = 0; t < RT; ++t) {
-          float cg[4] = {0.f, 0.f, 0.f, 0.f};
-          const uint32_t words[4] = {w[t].x, w[t].y, w[t].z, w[t].w};
+          for (int t = 0; t < RT; ++t) {
+            w[t] = wbuf[u][t];
+            sc[t] = sbuf[u][t];
+          }
+          load_group(grp + PF * WARPS, wbuf[u], sbuf[u]);
+          uint32_t b[4][2];
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            uint32_t a[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) a[j] = sub_bf16x2(((words[c] >> (4 * j)) & 0x000F000Fu) | 0x43004300u, 0x43084308u);
-            mma_bf16_16816(cg, a, b[c][0], b[c][1]);
+            b[c][0] = xrow[grp * 32 + c * 8];
+            b[c][1] = xrow[grp * 32 + c * 8 + 4];
           }
-          const float s_lo = __uint_as_float(sc[t] << 16), s_hi = __uint_as_float(sc[t] & 0xFFFF0000u);
-          acc[t][0] = fmaf(s_lo, cg[0], acc[t][0]);
-          acc[t][1] = fmaf(s_lo, cg[1], acc[t][1]);
-          acc[t][2] = fmaf(s_hi, cg[2], acc[t][2]);
-          acc[t][3] = fmaf(s_hi, cg[3], acc[t][3]);
+#pragma unroll
+          for (int t = 0; t < RT; ++t) {
+            // two accumulators per group (chunks 0, 1 and 2, 3): two independent chains of tensor-core instructions
+            float cg[2][4];
+            const uint32_t words[4] = {w[t].x, w[t].y, w[t].z, w[t].w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t a[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) a[j] = sub_bf16x2(((words[c] >> (4 * j)) & 0x000F000Fu) | 0x43004300u, 0x43084308u);
+              if (c & 1) mma_bf16_16816(cg[c >> 1], a, b[c][0], b[c][1], cg[c >> 1][0], cg[c >> 1][1], cg[c >> 1][2], cg[c >> 1][3]);
+              else mma_bf16_16816(cg[c >> 1], a, b[c][0], b[c][1], 0.f, 0.f, 0.f, 0.f);
+            }
+            const float s_lo = __uint_as_float(sc[t] << 16), s_hi = __uint_as_float(sc[t] & 0xFFFF0000u);
+            acc[t][0] = fmaf(s_lo, cg[0][0] + cg[1][0], acc[t][0]);
+            acc[t][1] = fmaf(s_lo, cg[0][1] + cg[1][1], acc[t][1]);
+            acc[t][2] = fmaf(s_hi, cg[0][2] + cg[1][2], acc[t][2]);
+            acc[t][3] = fmaf(s_hi, cg[0][3] + cg[1][3], acc[t][3]);
+          }
         }
       }
     }
-  }
 #pragma unroll
-  for (int t = 0; t < RT; ++t) {
-    float* r0 = red + ((size_t)(warp * RT * 16 + t * 16 + g) * 8 + 2 * tig);
-    r0[0] = acc[t][0];
-    r0[1] = acc[t][1];
-    r0[64] = acc[t][2];        // row g + 8
-    r0[65] = acc[t][3];
-  }
-  __syncthreads();
-  // thread -> (token, row of the CTA): a warp stores 32 consecutive outputs of one token
-  const int tok = tid >> 5, r = tid & 31;
-  const int row = tile0 * 16 + r;
-  if (tok < n && row < m) {
-    float sum = 0.f;
+    for (int t = 0; t < RT; ++t) {
+      float* r0 = red + ((size_t)(warp * RT * 16 + t * 16 + g) * 8 + 2 * tig);
+      r0[0] = acc[t][0];
+      r0[1] = acc[t][1];
+      r0[64] = acc[t][2];        // row g + 8
+      r0[65] = acc[t][3];
+    }
+    // the next tiles' first groups travel during the reduction
+    if (tile0 + RT < tile_end) {
+      tile0 += RT;
 #pragma unroll
-    for (int w = 0; w < WARPS; ++w) sum += red[(size_t)(w * RT * 16 + r) * 8 + tok];
-    if (f32_out) reinterpret_cast<float*>(Y)[(size_t)tok * ldy + row] = sum;
-    else reinterpret_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(sum);
+      for (int u = 0; u < PF; ++u) load_group(warp + u * WARPS, wbuf[u], sbuf[u]);
+      tile0 -= RT;
+    }
+    __syncthreads();
+    // thread -> (token, row of the CTA): a warp stores 32 consecutive outputs of one token
+    const int tok = tid >> 5, r = tid & 31;
+    const int row = tile0 * 16 + r;
+    if (tok < n && row < tile_end * 16) {
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) sum += red[(size_t)(w * RT * 16 + r) * 8 + tok];
+      if (f32_out) reinterpret_cast<float*>(Y)[(size_t)tok * ldy + row] = sum;
+      else reinterpret_cast<__nv_bfloat16*>(Y)[(size_t)tok * ldy + row] = __float2bfloat16_rn(sum);
+    }
+    __syncthreads();               // the partial sums are overwritten by the next tiles
   }
 }
 
@@ -289,7 +306,8 @@ int oq_adaln_linear(const void* X_bf16, int n_tokens, int ldx, const void* Wq, c
   if (ldx % 8 || !aligned16(X_bf16) || !aligned16(Wq) || !aligned16(scales))
     return fail(OQ_ERR_ALIGNMENT, "oq_adaln_linear: pointers must be 16-byte aligned and ldx a multiple of 8");
   const size_t red_bytes = (size_t)adaln::WARPS * adaln::RT * 16 * 8 * 4;
-  const size_t smem_max = (size_t)(n_tokens < adaln::MAXN ? n_tokens : adaln::MAXN) * (dim / 2 + 4) * 4 + red_bytes;
+  if ((long long)m * dim >= (1ll << 36)) return fail(OQ_ERR_UNSUPPORTED, "oq_adaln_linear: m * dim must be below 2^36");
+  const size_t smem_max = (size_t)((n_tokens < adaln::MAXN ? n_tokens : adaln::MAXN) + 1) * (dim / 2 + 4) * 4 + red_bytes;
   if (smem_max > 227 * 1024) return fail(OQ_ERR_UNSUPPORTED, "oq_adaln_linear: dim too large for the activation staging buffer");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   static bool attr_set = false;
@@ -298,15 +316,27 @@ int oq_adaln_linear(const void* X_bf16, int n_tokens, int ldx, const void* Wq, c
     if (e != cudaSuccess) return cuda_fail(e, "oq_adaln_linear (shared memory attribute)");
     attr_set = true;
   }
-  const int ctas = (m / 16 + adaln::RT - 1) / adaln::RT;
+  // one wave: as many CTAs as are resident at once, each with an equal share of the row tiles (a multiple of RT)
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaError_t ea = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (ea != cudaSuccess) return cuda_fail(ea, "cudaDeviceGetAttribute");
+  const int tiles = m / 16;
   const size_t ysz = y_dtype == OQ_F32 ? 4 : 2;
   // the tensor-core tile has 8 columns: more tokens than that take one pass over the weights per 8
   for (int n0 = 0; n0 < n_tokens; n0 += adaln::MAXN) {
     const int n = n_tokens - n0 < adaln::MAXN ? n_tokens - n0 : adaln::MAXN;
-    const size_t smem = (size_t)n * (dim / 2 + 4) * 4 + red_bytes;
+    const size_t smem = (size_t)(n + 1) * (dim / 2 + 4) * 4 + red_bytes;
+    int per_sm = 1;
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adaln::adaln_linear_kernel, adaln::THREADS, smem);
+    if (per_sm < 1) per_sm = 1;
+    const int slots = sms * per_sm;
+    int per_cta = (tiles + slots - 1) / slots;
+    per_cta = (per_cta + adaln::RT - 1) / adaln::RT * adaln::RT;
+    const int ctas = (tiles + per_cta - 1) / per_cta;
     adaln::adaln_linear_kernel<<<ctas, adaln::THREADS, smem, st>>>(
         reinterpret_cast<const uint4*>(Wq), reinterpret_cast<const uint32_t*>(scales),
-        reinterpret_cast<const __nv_bfloat16*>(X_bf16) + (size_t)n0 * ldx, n, ldx, m, dim,
+        reinterpret_cast<const __nv_bfloat16*>(X_bf16) + (size_t)n0 * ldx, n, ldx, m, dim, per_cta,
         reinterpret_cast<unsigned char*>(Y) + (size_t)n0 * ldy * ysz, ldy, y_dtype == OQ_F32 ? 1 : 0);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "oq_adaln_linear");
