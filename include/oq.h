@@ -178,6 +178,21 @@ int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out
  * OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
 int oq_device_status(int* status);
 
+/* ---- activations as bf16 levels ("decode once") ----------------------------------------------------- */
+
+/* An activation tile is used by every column tile of the output, so oq_qlinear decodes the same packed indices
+ * once per column tile.  These two calls decode them once per layer instead: oq_decode_levels writes
+ * out[row][k] = bf16(C[idx[row][k]]) (the level of Eq. 3, not yet multiplied by the norm) for a packed operand
+ * (device, rows x dim, the layout oq_rotate_quantize_act / oq_quantize_weights wrote) into out_bf16 (device,
+ * [rows][ldo], ldo >= dim, ldo % 8 == 0, 16-byte aligned); oq_qlinear_levels is oq_qlinear with that matrix as the
+ * activation operand (fetched by TMA) and all decoding warps on the weights.  Same bf16 operands, same order of
+ * accumulation: Y is bit-identical to oq_qlinear's.  dim % 128 == 0, m % 8 == 0, weight bits 2..4; other
+ * arguments, asynchrony and errors as for oq_qlinear. */
+int oq_decode_levels(const void* idx, int rows, int dim, const oq_codebook* cb, void* out_bf16, int ldo, void* stream);
+int oq_qlinear_levels(const void* Xd_bf16, int ldxd, const float* Xq_norm, int n_tokens, const void* Wq_idx,
+                      const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y, int ldy, int y_dtype,
+                      void* stream);
+
 /* ---- AdaLN modulation projections (weight-only INT4, bf16 activations) ----------------------------- */
 
 /* The AdaLN modulation projections are not rotated: their weights are quantized to INT4 by round-to-nearest in

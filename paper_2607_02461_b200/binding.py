@@ -51,6 +51,8 @@ def lib():
             "oq_selftest_bounded_wait": (i, [vp]),
             "oq_debug_select_rq_kernel": (i, [i]),
             "oq_rq_plan": (i, [vp, vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(sz)]),
+            "oq_decode_levels": (i, [vp, i, i, vp, vp, i, vp]),
+            "oq_qlinear_levels": (i, [vp, i, vp, i, vp, vp, i, vp, i, vp, i, i, vp]),
             "oq_adaln_packed_bytes": (i, [i, i, C.POINTER(sz), C.POINTER(sz)]),
             "oq_adaln_quantize_weights": (i, [vp, i, i, i, vp, vp, vp]),
             "oq_adaln_linear": (i, [vp, i, i, vp, vp, i, i, vp, i, i, vp]),
@@ -231,6 +233,28 @@ def oq_rq_plan(rot, cb):
 
 def oq_debug_select_rq_kernel(which):
     _check(lib().oq_debug_select_rq_kernel(int(which)))
+
+
+def oq_decode_levels(idx, rows, dim, cb, out=None):
+    """Packed indices [rows, pitch] -> bf16 levels [rows, dim] (written once, read by oq_qlinear_levels)."""
+    import torch
+    if out is None:
+        out = torch.empty((rows, dim), dtype=torch.bfloat16, device=idx.device)
+    _check(lib().oq_decode_levels(_ptr(idx), rows, dim, cb.handle, _ptr(out), out.stride(0) if rows > 1 else dim, _stream()))
+    return out
+
+
+def oq_qlinear_levels(Xd, Xq_norm, Wq_idx, Wq_norm, cb_w, dim, out=None, out_dtype=None):
+    """oq_qlinear with the activations given as bf16 levels [N, dim]."""
+    import torch
+    n, m = Xd.shape[0], Wq_idx.shape[0]
+    if out is None:
+        out = torch.empty((n, m), dtype=out_dtype or torch.bfloat16, device=Xd.device)
+    ydt = OQ_F32 if out.dtype == torch.float32 else OQ_BF16
+    _check(lib().oq_qlinear_levels(_ptr(Xd), Xd.stride(0) if n > 1 else dim, _ptr(Xq_norm), n, _ptr(Wq_idx),
+                                   _ptr(Wq_norm), m, cb_w.handle, dim, _ptr(out), out.stride(0) if n > 1 else m, ydt,
+                                   _stream()))
+    return out
 
 
 def oq_adaln_packed_bytes(m, dim):

@@ -5,8 +5,17 @@
 // with byte-permute table look-ups, written into shared memory in the tensor core's K-major
 // 128-byte-swizzled layout, and contracted with tcgen05.mma.cta_group::2 (fp32 accumulators in tensor
 // memory, two SMs per 256 x 256 tile).  Every device-side wait is bounded and reports to a status word.
+//
+// The activation operand comes in one of two forms: packed indices, decoded here like the weights (BITS_A = 2, 3,
+// 4), or the bf16 levels C_a[idx] written out once by the producer (BITS_A = 0).  An activation tile is used by
+// every column tile of the output, so decoding it once per layer instead of once per tile takes half of the decode
+// work out of this kernel: the tiles then arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle, no SM
+// instructions), and all 16 decoding warps work on the weights.  Both forms feed the same bf16 values to the same
+// MMAs in the same order: the outputs are bit-identical.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
+#include "oq_decode.cuh"
 #include "oq_internal.h"
 #include "oq_sm100.cuh"
 
@@ -18,113 +27,6 @@ constexpr int BK = 64;                  // coordinates per swizzle atom: 64 bf16
 constexpr int DECODE_THREADS = 512;    // 16 decoding warps per CTA
 constexpr int TMEM_COLS = 512;         // two 128 x 256 fp32 accumulators per CTA
 
-// Byte tables of the positive levels: lo/hi bytes of bf16(c_j), j = magnitude rank.
-struct Tables {
-  uint32_t lo0, lo1, hi0, hi1;
-};
-__device__ __forceinline__ Tables make_tables(const CodebookParams& cb) {
-  const int M = (1 << cb.bits) >> 1;
-  Tables t = {0u, 0u, 0u, 0u};
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const uint32_t v = j < M ? cb.level_bf16[M + j] : 0u;
-    if (j < 4) {
-      t.lo0 |= (v & 0xFFu) << (8 * j);
-      t.hi0 |= (v >> 8) << (8 * j);
-    } else {
-      t.lo1 |= (v & 0xFFu) << (8 * (j - 4));
-      t.hi1 |= (v >> 8) << (8 * (j - 4));
-    }
-  }
-  return t;
-}
-
-// Decodes 32 consecutive coordinates (BITS words of one packed row) into four 16-byte chunks of bf16.
-// Raw packed words of 32 coordinates of one row (BITS words), fetched ahead of their use.
-template <int BITS>
-struct Raw {
-  uint32_t w[BITS];
-};
-template <int BITS>
-__device__ __forceinline__ Raw<BITS> load_raw(const uint32_t* __restrict__ src) {
-  Raw<BITS> r;
-  if (BITS == 4) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
-    r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[BITS - 1] = v.w;
-  } else if (BITS == 3) {
-    r.w[0] = __ldg(src); r.w[1] = __ldg(src + 1); r.w[2] = __ldg(src + 2);
-  } else {
-    const uint2 v = __ldg(reinterpret_cast<const uint2*>(src));
-    r.w[0] = v.x; r.w[1] = v.y;
-  }
-  return r;
-}
-
-// The 2 * BITS contiguous words of 64 coordinates of one row, as two 32-coordinate pieces.
-template <int BITS>
-__device__ __forceinline__ void load_raw64(const uint32_t* __restrict__ src, Raw<BITS>& a, Raw<BITS>& b) {
-  if (BITS == 4) {          // 32 bytes, 16-byte aligned
-    a = load_raw<BITS>(src);
-    b = load_raw<BITS>(src + 4);
-  } else if (BITS == 3) {   // 24 bytes, 8-byte aligned
-    const uint2 v0 = __ldg(reinterpret_cast<const uint2*>(src));
-    const uint2 v1 = __ldg(reinterpret_cast<const uint2*>(src) + 1);
-    const uint2 v2 = __ldg(reinterpret_cast<const uint2*>(src) + 2);
-    a.w[0] = v0.x; a.w[1] = v0.y; a.w[BITS - 1] = v1.x;
-    b.w[0] = v1.y; b.w[1] = v2.x; b.w[BITS - 1] = v2.y;
-  } else {                  // 16 bytes, 16-byte aligned
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
-    a.w[0] = v.x; a.w[1] = v.y;
-    b.w[0] = v.z; b.w[1] = v.w;
-  }
-}
-
-template <int BITS>
-__device__ __forceinline__ void decode32(const Raw<BITS>& raw, const Tables& t, uint4 out[4]) {
-  if (BITS == 4) {
-    const uint32_t* w = raw.w;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint32_t sel = w[q] & 0x77777777u;
-      const uint32_t loA = prmt(t.lo0, t.lo1, sel), loB = prmt(t.lo0, t.lo1, sel >> 16);
-      const uint32_t hiA = prmt(t.hi0, t.hi1, sel) ^ (w[q] & 0x80808080u);
-      const uint32_t hiB = prmt(t.hi0, t.hi1, sel >> 16) ^ ((w[q] << 4) & 0x80808080u);
-      out[q] = make_uint4(prmt(loA, hiA, 0x5140u), prmt(loA, hiA, 0x7362u), prmt(loB, hiB, 0x5140u),
-                          prmt(loB, hiB, 0x7362u));
-    }
-  } else {
-    const uint32_t mw[2] = {raw.w[0], raw.w[BITS == 3 ? 1 : 0]};
-    const uint32_t s = raw.w[BITS - 1];
-    // byte-permute selectors of the 8 groups of 4 coordinates: the permute reads only the low 16 bits of a
-    // selector, so one mask serves two groups (the second after a shift by 16)
-    uint32_t selv[8];
-    if (BITS == 3) {
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const uint32_t e = mw[u] & 0x33333333u, o = (mw[u] >> 2) & 0x33333333u;
-        selv[4 * u] = e; selv[4 * u + 1] = o; selv[4 * u + 2] = e >> 16; selv[4 * u + 3] = o >> 16;
-      }
-    } else {
-#pragma unroll
-      for (int g = 0; g < 4; ++g) {
-        const uint32_t e = (mw[0] >> g) & 0x11111111u;
-        selv[g] = e; selv[4 + g] = e >> 16;
-      }
-    }
-    uint32_t r[16];
-#pragma unroll
-    for (int G = 0; G < 8; ++G) {
-      const uint32_t sel = selv[G];
-      const uint32_t lo = prmt(t.lo0, t.lo0, sel);
-      const uint32_t hi = prmt(t.hi0, t.hi0, sel) ^ ((s << G) & 0x80808080u);
-      r[2 * G] = prmt(lo, hi, 0x5140u);
-      r[2 * G + 1] = prmt(lo, hi, 0x7362u);
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) out[q] = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-  }
-}
-
 // ---------------------------------------------------------------------------------------------------------
 namespace pair {
 constexpr int PSTAGES = 3;
@@ -133,7 +35,7 @@ constexpr uint32_t ATOM_BYTES = 128 * BK * 2;                          // 128 ro
 constexpr uint32_t PA_BYTES = 2 * ATOM_BYTES, PB_BYTES = 2 * ATOM_BYTES;
 constexpr uint32_t PSTAGE_BYTES = PA_BYTES + PB_BYTES;                 // 64 KB
 constexpr int EPI_THREADS = 128;
-constexpr int PTHREADS = DECODE_THREADS + EPI_THREADS + 32;   // 16 decode warps, 4 epilogue warps, 1 MMA warp
+constexpr int PTHREADS = DECODE_THREADS + EPI_THREADS + 64;   // 16 decode warps, 4 epilogue warps, 1 MMA warp, 1 TMA warp
 constexpr size_t PSMEM_BYTES = PSTAGES * PSTAGE_BYTES + 1024 + 256;
 }  // namespace pair
 
@@ -179,6 +81,79 @@ __device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void commit_multicast(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
+// Address of the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  return ra;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+// One box of the activation matrix (64 coordinates x 128 rows, 128-byte swizzle) into this CTA's shared memory; the
+// bytes are counted on a barrier of the pair's leading CTA (never a multicast: each CTA fetches its own rows).
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t cluster_bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y) : "memory");
+}
+
+// Weight decode loop of the kernel whose activations arrive as bf16 levels: all 512 decoding threads work on this
+// CTA's 128 weight rows.  Warps 0-7 fill swizzle atom 0 of a stage, warps 8-15 atom 1; inside an atom a thread owns
+// (row t2/2, 32-coordinate half t2%2): one load of BITS words (adjacent lanes read adjacent pieces), four 16-byte
+// stores; the 8 lanes of a quarter warp hit 8 different chunk positions, i.e. all 32 banks.
+template <int BITS>
+__device__ __forceinline__ void dense_b_decode_loop(const uint32_t* __restrict__ packed, int nrows, int dim, const Tables& t,
+                                                    unsigned char* smem, uint32_t full0, uint32_t empty0, int tid512,
+                                                    uint32_t rank, int pair_id, int npairs, int ntiles, int tiles_m,
+                                                    int kblocks, volatile int* abort_flag, int* status) {
+  using namespace pair;
+  const int lane = threadIdx.x & 31;
+  const int atom = tid512 >> 8, t2 = tid512 & 255, row = t2 >> 1, half = t2 & 1;
+  const int pitch = dim / 32 * BITS;
+  unsigned char* const tile0 = smem + PA_BYTES + (uint32_t)atom * ATOM_BYTES + (uint32_t)row * 128u;
+  const uint32_t rx = (uint32_t)(row & 7) << 4, c0b = (uint32_t)half * 64u;
+  uint32_t st = 0, ph = 0;
+  bool first_round = true;
+  Raw<BITS> nxt;                                      // packed words of the NEXT stage
+  int f_tile = pair_id, f_kb = 0;
+  const uint32_t* fsrc = nullptr;
+  auto set_fetch_tile = [&](int tile) {
+    const int r0 = (tile % tiles_m) * 256 + (int)rank * 128;     // column tiles vary fastest (see the kernel)
+    fsrc = packed + (size_t)min(r0 + row, nrows - 1) * pitch + (atom * 2 + half) * BITS;   // rows past the end re-read the last
+  };
+  auto fetch_next = [&]() {
+    if (f_tile >= ntiles) return;
+    nxt = load_raw<BITS>(fsrc);
+    fsrc += 4 * BITS;                                 // 128 coordinates per stage
+    if (++f_kb == kblocks) {
+      f_kb = 0;
+      f_tile += npairs;
+      if (f_tile < ntiles) set_fetch_tile(f_tile);
+    }
+  };
+  if (f_tile < ntiles) set_fetch_tile(f_tile);
+  fetch_next();
+  for (int tile = pair_id; tile < ntiles; tile += npairs) {
+    for (int kb = 0; kb < kblocks; ++kb) {
+      const Raw<BITS> cur = nxt;
+      fetch_next();
+      if (!first_round) {
+        if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
+        __syncwarp();
+      }
+      unsigned char* Ss = tile0 + st * PSTAGE_BYTES;
+      uint4 v[4];
+      decode32<BITS>(cur, t, v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ((c0b + ((uint32_t)q << 4)) ^ rx)) = v[q];
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(full0 + 8 * st, 0);          // to CTA 0, where the MMAs are issued
+      if (++st == PSTAGES) { st = 0; ph ^= 1; first_round = false; }
+    }
+  }
 }
 
 // Decode loop of one thread of the two-SM kernel: the thread owns one (row, 32-coordinate half) of this CTA's
@@ -266,7 +241,8 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
 
 template <int BITS_A, int BITS_W, bool F32_OUT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::PTHREADS, 1)
-qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm, int n_tokens,
+qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* __restrict__ Aq,
+                    const float* __restrict__ a_norm, int n_tokens,
                     const uint32_t* __restrict__ Wq, const __nv_bfloat16* __restrict__ w_norm, int m, int dim,
                     CodebookParams cba, CodebookParams cbw, void* __restrict__ Y, int ldy, int* status) {
   using namespace pair;
@@ -282,11 +258,13 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
   const uint32_t rank = cluster_ctarank();
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + PSTAGES);
   const uint32_t accfull0 = smem_u32(bars + 2 * PSTAGES), accempty0 = smem_u32(bars + 2 * PSTAGES + 2);
-  constexpr int MMA_WARP = (DECODE_THREADS + EPI_THREADS) / 32;
+  constexpr int MMA_WARP = (DECODE_THREADS + EPI_THREADS) / 32, TMA_WARP = MMA_WARP + 1;
+  constexpr bool DENSE_A = BITS_A == 0;               // activations as bf16 levels, fetched by TMA
 
   if (tid == 0) {
     for (int s = 0; s < PSTAGES; ++s) {
-      mbar_init(full0 + 8 * s, 2 * (DECODE_THREADS / 32));   // one arrival per decoding warp of BOTH CTAs (used in CTA 0)
+      // one arrival per decoding warp of BOTH CTAs (used in CTA 0); with TMA also one per CTA that announces its bytes
+      mbar_init(full0 + 8 * s, 2 * (DECODE_THREADS / 32) + (DENSE_A ? 2 : 0));
       mbar_init(empty0 + 8 * s, 1);                          // multicast commit
     }
     for (int b = 0; b < 2; ++b) {
@@ -314,7 +292,11 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
 
   const int kblocks = dim / PBK;
   const int tiles_n = (n_tokens + 255) / 256;
-  const int ntiles = tiles_n * ((m + 255) / 256);
+  const int tiles_m = (m + 255) / 256;
+  const int ntiles = tiles_n * tiles_m;
+  // Tile order.  Packed activations: row tiles vary fastest (the pairs running together share a weight tile).  bf16
+  // levels: column tiles vary fastest, so that the pairs running together share activation tiles, which are four
+  // times larger than packed ones and may not fit in L2 as a whole.
   const int npairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
 
   if (warp == MMA_WARP) {
@@ -347,13 +329,39 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
         commit_multicast(accfull0 + 8 * buf);      // both CTAs' epilogue warps may read accumulator `buf`
       }
     }
+  } else if (warp == TMA_WARP) {
+    // ------------------------------- activation tiles by TMA: one thread per CTA -------------------------------
+    if (DENSE_A && lane == 0) {
+      const uint32_t full_leader = map_to_cta(full0, 0);
+      uint32_t st = 0, ph = 0;
+      bool first_round = true;
+      for (int tile = pair_id; tile < ntiles && !*abort_flag; tile += npairs) {
+        const int n0 = (tile / tiles_m) * 256 + (int)rank * 128;       // rows past the last token read as zeros
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!first_round) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
+          if (*abort_flag) break;
+          mbar_arrive_expect_tx_cluster(full_leader + 8 * st, PA_BYTES);
+          const uint32_t dst = smem_u32(smem + st * PSTAGE_BYTES);
+          tma_load_box(dst, &tmap_a, kb * PBK, n0, full_leader + 8 * st);
+          tma_load_box(dst + ATOM_BYTES, &tmap_a, kb * PBK + BK, n0, full_leader + 8 * st);
+          if (++st == PSTAGES) { st = 0; ph ^= 1; first_round = false; }
+        }
+      }
+      // after a wait gave up somewhere, tiles requested above may still be on their way into this CTA's shared memory:
+      // give them time to land before the CTA ends (they complete within microseconds)
+      if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) {}
+      }
+    }
   } else if (warp >= DECODE_THREADS / 32) {
     // ------------------------------- epilogue warps (4 per CTA) -------------------------------
     const int q = warp & 3;                          // TMEM lane quarter of this warp
     uint32_t lt = 0;
     for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
       const uint32_t buf = lt & 1;
-      const int n0 = (tile % tiles_n) * 256 + (int)rank * 128, i0 = (tile / tiles_n) * 256;
+      const int n0 = (DENSE_A ? tile / tiles_m : tile % tiles_n) * 256 + (int)rank * 128;
+      const int i0 = (DENSE_A ? tile % tiles_m : tile / tiles_n) * 256;
       if (lane == 0) mbar_wait(accfull0 + 8 * buf, (lt >> 1) & 1, abort_flag, status, WAIT_ACC_FULL);
       __syncwarp();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -398,10 +406,14 @@ qlinear_pair_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a
     }
   } else {
     // ------------------------------- decoders (16 warps per CTA) -------------------------------
-    // threads 0-255: this CTA's 128 rows of A; threads 256-511: its 128 rows of B
-    if (tid < 256) {
+    // threads 0-255: this CTA's 128 rows of A; threads 256-511: its 128 rows of B (all 512 on B when A comes by TMA)
+    if constexpr (DENSE_A) {
+      const Tables tw = make_tables(cbw);
+      dense_b_decode_loop<BITS_W>(Wq, m, dim, tw, smem, full0, empty0, tid, rank, pair_id, npairs, ntiles, tiles_m,
+                                  kblocks, abort_flag, status);
+    } else if (tid < 256) {
       const Tables ta = make_tables(cba);
-      pair_decode_loop<BITS_A, true>(Aq, n_tokens, dim, ta, smem, full0, empty0, tid, rank, pair_id, npairs, ntiles,
+      pair_decode_loop<(DENSE_A ? 4 : BITS_A), true>(Aq, n_tokens, dim, ta, smem, full0, empty0, tid, rank, pair_id, npairs, ntiles,
                                      tiles_n, kblocks, abort_flag, status);
     } else {
       const Tables tw = make_tables(cbw);
@@ -429,8 +441,53 @@ __global__ void bounded_wait_probe_kernel(int* status, long long max_cycles) {
   }
 }
 
+// Writes an operand out as bf16 levels: thread = 32 consecutive coordinates of one row.
+template <int BITS>
+__global__ void decode_levels_kernel(const uint32_t* __restrict__ packed, int rows, int dim, CodebookParams cb,
+                                     __nv_bfloat16* __restrict__ out, int ldo) {
+  const Tables t = make_tables(cb);
+  const int per_row = dim / 32, pitch = per_row * BITS;
+  const long long total = (long long)rows * per_row;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const int row = (int)(i / per_row), c = (int)(i - (long long)row * per_row);
+    const Raw<BITS> raw = load_raw<BITS>(packed + (size_t)row * pitch + c * BITS);
+    uint4 v[4];
+    decode32<BITS>(raw, t, v);
+    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)row * ldo + c * 32);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) dst[q] = v[q];
+  }
+}
+
+// Tensor map of a row-major bf16 matrix [rows][ld] for boxes of 64 coordinates x 128 rows with the 128-byte swizzle
+// (the driver entry point is looked up once; no link-time dependency on the driver library).
+cudaError_t make_levels_map(const void* base, int rows, int dim, int ld, CUtensorMap* map) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    encode = reinterpret_cast<EncodeFn>(fn);
+  }
+  const cuuint64_t gdim[2] = {(cuuint64_t)dim, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, 128u};
+  const cuuint32_t estride[2] = {1u, 1u};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estride,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 template <int BA, int BW, bool F32>
-cudaError_t launch_pair(int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
+cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
                         const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw,
                         void* Y, int ldy, int* status) {
   auto k = qlinear_pair_kernel<BA, BW, F32>;
@@ -455,16 +512,27 @@ cudaError_t launch_pair(int sms, cudaStream_t st, const uint32_t* Aq, const floa
   int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev] : sms / 2;
   if (pairs > sms / 2) pairs = sms / 2;
   if (pairs > ntiles) pairs = ntiles;
-  return launch_dependent(k, 2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
+  return launch_dependent(k, 2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st, tmap, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
 }
 
 template <int BA, int BW>
 int launch_bits(bool f32, int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
                 const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw, void* Y,
                 int ldy, int* status) {
-  const cudaError_t e = f32 ? launch_pair<BA, BW, true>(sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status)
-                            : launch_pair<BA, BW, false>(sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
+  static const CUtensorMap no_map = {};
+  const cudaError_t e = f32 ? launch_pair<BA, BW, true>(no_map, sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status)
+                            : launch_pair<BA, BW, false>(no_map, sms, st, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
   if (e != cudaSuccess) return cuda_fail(e, "oq_qlinear launch");
+  return OQ_OK;
+}
+
+// Activations as bf16 levels (fetched by TMA through `tmap`).
+template <int BW>
+int launch_levels_bits(const CUtensorMap& tmap, bool f32, int sms, cudaStream_t st, const float* an, int n, const uint32_t* Wq,
+                       const __nv_bfloat16* wn, int m, int dim, const CodebookParams& cw, void* Y, int ldy, int* status) {
+  const cudaError_t e = f32 ? launch_pair<0, BW, true>(tmap, sms, st, nullptr, an, n, Wq, wn, m, dim, cw, cw, Y, ldy, status)
+                            : launch_pair<0, BW, false>(tmap, sms, st, nullptr, an, n, Wq, wn, m, dim, cw, cw, Y, ldy, status);
+  if (e != cudaSuccess) return cuda_fail(e, "oq_qlinear_levels launch");
   return OQ_OK;
 }
 
@@ -511,6 +579,85 @@ int qlinear_launch(const void* Xq_idx, const float* Xq_norm, int n_tokens, const
 }
 
 }  // namespace oq
+
+namespace oq {
+
+int qlinear_levels_launch(const void* Xd_bf16, int ldxd, const float* Xq_norm, int n_tokens, const void* Wq_idx,
+                          const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y, int ldy, int y_dtype,
+                          int* status, void* stream) {
+  if (!cb_w) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: NULL codebook");
+  if (n_tokens < 0 || m < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: bad sizes");
+  if (cb_w->dim != dim) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: codebook dim differs from dim");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, "oq_qlinear_levels: dim must be a multiple of 128");
+  if (m % 8) return fail(OQ_ERR_UNSUPPORTED, "oq_qlinear_levels: m must be a multiple of 8");
+  if (y_dtype != OQ_BF16 && y_dtype != OQ_F32) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: unknown y_dtype");
+  const int bw = cb_w->bits;
+  if (bw < 2 || bw > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_qlinear_levels: weight bits must be 2, 3 or 4");
+  if (n_tokens == 0 || m == 0) return OQ_OK;
+  if (!Xd_bf16 || !Xq_norm || !Wq_idx || !Wq_norm_bf16 || !Y) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: NULL buffer");
+  if (ldy < m || ldxd < dim) return fail(OQ_ERR_INVALID_ARG, "oq_qlinear_levels: leading dimension too small");
+  if (ldy % 8 || ldxd % 8 || !aligned16(Xd_bf16) || !aligned16(Wq_idx) || !aligned16(Y) || !aligned16(Wq_norm_bf16))
+    return fail(OQ_ERR_ALIGNMENT, "oq_qlinear_levels: pointers must be 16-byte aligned and leading dimensions multiples of 8");
+  if (!status) status = device_status_word();
+  if (!status) return fail(OQ_ERR_CUDA, "oq_qlinear_levels: cannot allocate the device status word");
+  CUtensorMap tmap;
+  cudaError_t ce = make_levels_map(Xd_bf16, n_tokens, dim, ldxd, &tmap);
+  if (ce != cudaSuccess) return cuda_fail(ce, "oq_qlinear_levels: tensor map");
+  const CodebookParams cw = codebook_params(cb_w);
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (ce != cudaSuccess) return cuda_fail(ce, "cudaDeviceGetAttribute");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const uint32_t* W = reinterpret_cast<const uint32_t*>(Wq_idx);
+  const __nv_bfloat16* wn = reinterpret_cast<const __nv_bfloat16*>(Wq_norm_bf16);
+  const bool f32 = y_dtype == OQ_F32;
+  if (bw == 4) return launch_levels_bits<4>(tmap, f32, sms, st, Xq_norm, n_tokens, W, wn, m, dim, cw, Y, ldy, status);
+  if (bw == 3) return launch_levels_bits<3>(tmap, f32, sms, st, Xq_norm, n_tokens, W, wn, m, dim, cw, Y, ldy, status);
+  return launch_levels_bits<2>(tmap, f32, sms, st, Xq_norm, n_tokens, W, wn, m, dim, cw, Y, ldy, status);
+}
+
+int decode_levels_launch(const void* idx, int rows, int dim, const oq_codebook* cb, void* out_bf16, int ldo, void* stream) {
+  if (!cb) return fail(OQ_ERR_INVALID_ARG, "oq_decode_levels: NULL codebook");
+  if (rows < 0 || dim <= 0 || cb->dim != dim) return fail(OQ_ERR_INVALID_ARG, "oq_decode_levels: bad sizes");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, "oq_decode_levels: dim must be a multiple of 128");
+  if (cb->bits < 2 || cb->bits > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_decode_levels: bits must be 2, 3 or 4");
+  if (rows == 0) return OQ_OK;
+  if (!idx || !out_bf16) return fail(OQ_ERR_INVALID_ARG, "oq_decode_levels: NULL buffer");
+  if (ldo < dim) return fail(OQ_ERR_INVALID_ARG, "oq_decode_levels: ldo smaller than dim");
+  if (ldo % 8 || !aligned16(idx) || !aligned16(out_bf16))
+    return fail(OQ_ERR_ALIGNMENT, "oq_decode_levels: pointers must be 16-byte aligned and ldo a multiple of 8");
+  const CodebookParams cp = codebook_params(cb);
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  const long long total = (long long)rows * (dim / 32);
+  long long blocks = (total + 255) / 256;
+  if (blocks > (long long)sms * 8) blocks = (long long)sms * 8;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const uint32_t* p = reinterpret_cast<const uint32_t*>(idx);
+  __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out_bf16);
+  if (cb->bits == 4) e = launch_dependent(decode_levels_kernel<4>, (int)blocks, 256, 0, st, p, rows, dim, cp, o, ldo);
+  else if (cb->bits == 3) e = launch_dependent(decode_levels_kernel<3>, (int)blocks, 256, 0, st, p, rows, dim, cp, o, ldo);
+  else e = launch_dependent(decode_levels_kernel<2>, (int)blocks, 256, 0, st, p, rows, dim, cp, o, ldo);
+  if (e != cudaSuccess) return cuda_fail(e, "oq_decode_levels");
+  return OQ_OK;
+}
+
+}  // namespace oq
+
+extern "C" int oq_qlinear_levels(const void* Xd_bf16, int ldxd, const float* Xq_norm, int n_tokens, const void* Wq_idx,
+                                 const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y, int ldy,
+                                 int y_dtype, void* stream) {
+  return oq::qlinear_levels_launch(Xd_bf16, ldxd, Xq_norm, n_tokens, Wq_idx, Wq_norm_bf16, m, cb_w, dim, Y, ldy, y_dtype,
+                                   nullptr, stream);
+}
+
+extern "C" int oq_decode_levels(const void* idx, int rows, int dim, const oq_codebook* cb, void* out_bf16, int ldo,
+                                void* stream) {
+  return oq::decode_levels_launch(idx, rows, dim, cb, out_bf16, ldo, stream);
+}
 
 extern "C" int oq_selftest_bounded_wait(void* stream) {
   int* status = oq::device_status_word();

@@ -54,7 +54,7 @@ def run_rq(n, d, bits, block, iters):
             "ms_min": best, "bytes": nbytes, "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
 
 
-def run_gemm(n, d, m, ba, bw, iters):
+def run_gemm(n, d, m, ba, bw, iters, levels=False):
     rot = B.oq_make_rpbh(d, 128, 0)
     cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
     xq, xs = B.oq_rotate_quantize_act(gen_x(n, d), rot, cba)
@@ -62,9 +62,13 @@ def run_gemm(n, d, m, ba, bw, iters):
     wq, wr = B.oq_quantize_weights(W, rot, cbw)
     del W
     Y = torch.empty((n, m), dtype=torch.bfloat16, device="cuda")
-    med, best = time_kernel(lambda: B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out=Y), iters)
+    if levels:
+        xd = B.oq_decode_levels(xq, n, d, cba)
+        med, best = time_kernel(lambda: B.oq_qlinear_levels(xd, xs, wq, wr, cbw, d, out=Y), iters)
+    else:
+        med, best = time_kernel(lambda: B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out=Y), iters)
     fl = 2.0 * n * m * d
-    return {"kernel": "qlinear", "tokens": n, "dim": d, "m": m, "bits_a": ba, "bits_w": bw, "ms_median": med,
+    return {"kernel": "qlinear_levels" if levels else "qlinear", "tokens": n, "dim": d, "m": m, "bits_a": ba, "bits_w": bw, "ms_median": med,
             "ms_min": best, "flops": fl, "tflops": fl / med / 1e9, "tflops_best": fl / best / 1e9}
 
 
@@ -93,6 +97,7 @@ def main(argv=None):
     ap.add_argument("--block", type=int, default=128)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--levels", action="store_true", help="gemm: activations as bf16 levels (oq_qlinear_levels)")
     ap.add_argument("--kernel", type=int, default=0, help="rotate+quantize kernel: 0 auto, 1 general, 2 registers, 3 tensor cores")
     a = ap.parse_args(argv)
     oqbuild.build()
@@ -100,7 +105,7 @@ def main(argv=None):
     if a.mode == "rq":
         print(json.dumps(run_rq(a.tokens, a.dim, a.bits, a.block, a.iters)))
     elif a.mode == "gemm":
-        print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters)))
+        print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters, a.levels)))
     elif a.mode == "adaln":
         print(json.dumps(run_adaln(a.tokens, a.dim, a.m, a.iters)))
     else:

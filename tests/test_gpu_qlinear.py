@@ -170,3 +170,32 @@ def test_back_to_back_launches_into_shared_buffers_match_serialised_runs():
     assert B.oq_device_status() == 0
     for a, b in zip(ref, got):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("bits_a,bits_w", [(4, 4), (3, 3), (4, 2), (2, 3)])
+@pytest.mark.parametrize("n,m,d", [(200, 520, 2048), (1, 8, 128), (257, 264, 384), (1000, 1536, 3072)])
+def test_levels_form_is_bit_identical_to_packed_form(n, m, d, bits_a, bits_w):
+    """Activations written out once as bf16 levels and fetched by TMA: same operands, same accumulation order, so the
+    same output bits as the kernel that decodes the packed activations itself; the level matrix itself is the
+    codebook's bf16 table indexed by the unpacked indices."""
+    import torch
+    rot = B.oq_make_rpbh(d, 128, 0)
+    cba, cbw = B.oq_build_codebook(d, bits_a), B.oq_build_codebook(d, bits_w)
+    xb, wb = synth.activations(n, d, seed=3100 + n), synth.weights(m, d, seed=3200 + m)
+    xq, xs = B.oq_rotate_quantize_act(_dev(xb), rot, cba)
+    wq, wr = B.oq_quantize_weights(_dev(wb), rot, cbw)
+    xd = B.oq_decode_levels(xq, n, d, cba)
+    idx = B.oq_unpack_indices(xq, n, d, bits_a).cpu().numpy()
+    levels_bits = obf.f64_to_bf16_bits(ocb.lloyd_max(d, bits_a).centroids)
+    assert np.array_equal(xd.view(torch.int16).cpu().numpy().view(np.uint16), levels_bits[idx])
+    for dt in (torch.bfloat16, torch.float32):
+        ref = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out_dtype=dt)
+        got = B.oq_qlinear_levels(xd, xs, wq, wr, cbw, d, out_dtype=dt)
+        torch.cuda.synchronize()
+        assert B.oq_device_status() == 0
+        assert torch.equal(ref, got)
+    # a level matrix with a leading dimension larger than dim
+    wide = torch.zeros((n, d + 64), dtype=torch.bfloat16, device="cuda")
+    B.oq_decode_levels(xq, n, d, cba, out=wide[:, :d])
+    got = B.oq_qlinear_levels(wide[:, :d], xs, wq, wr, cbw, d)
+    assert torch.equal(got, B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d))
