@@ -54,7 +54,8 @@ typedef struct oq_rpbh oq_rpbh;         /* RPBH rotation Pi_d: permutation + sig
 
 /* Lloyd-Max codebook of 2^bits levels for the coordinate marginal f_dim of a random unit vector
  * (Eq. 2: f_d(t) ~ (1 - t^2)^((d-3)/2) on [-1,1]; Eq. 3: nearest-level map).  The exact f_dim is used,
- * not its Gaussian approximation.  dim >= 16, bits in 1..4.  *out is owned by the caller
+ * not its Gaussian approximation.  dim >= 16, bits in 1..4 or 6 (6: activations only, see
+ * oq_rotate_quantize_act_levels; takes a few seconds).  *out is owned by the caller
  * (oq_codebook_destroy).  Errors: OQ_ERR_INVALID_ARG, OQ_ERR_UNSUPPORTED. */
 int oq_build_codebook(int dim, int bits, oq_codebook** out);
 
@@ -192,6 +193,18 @@ int oq_decode_levels(const void* idx, int rows, int dim, const oq_codebook* cb, 
 int oq_qlinear_levels(const void* Xd_bf16, int ldxd, const float* Xq_norm, int n_tokens, const void* Wq_idx,
                       const void* Wq_norm_bf16, int m, const oq_codebook* cb_w, int dim, void* Y, int ldy, int y_dtype,
                       void* stream);
+
+/* 6-bit activations (the W4A6 setting of the video models, Sec. 5.1): 64 levels do not fit the byte-permute decode
+ * of oq_qlinear, so the rotate+quantize pass writes the levels themselves: Xd_bf16[n][k] = bf16(C_a[idx[n][k]])
+ * (device, [n_tokens][ldxd], ldxd >= dim, ldxd % 8 == 0, 16-byte aligned), the operand of oq_qlinear_levels, and
+ * Xq_norm[n] = s (fp32) as oq_rotate_quantize_act does.  cb_a must have 6 bits (oq_build_codebook(dim, 6)); the
+ * nearest level is found on a uniform grid of 256 cells over the normalised magnitude, each holding at most one
+ * boundary (same rule as Eq. 3 with ties to the lower index).  idx_u8: optional device [n_tokens][dim] bytes that
+ * receive the level indices 0..63 (16-byte aligned; NULL to skip); dbg_rotated as in oq_rotate_quantize_act.
+ * Hadamard blocks of 64..4096.  Errors as for oq_rotate_quantize_act. */
+int oq_rotate_quantize_act_levels(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                                  const oq_codebook* cb_a, void* Xd_bf16, int ldxd, float* Xq_norm, void* idx_u8,
+                                  float* dbg_rotated, void* stream);
 
 /* ---- AdaLN modulation projections (weight-only INT4, bf16 activations) ----------------------------- */
 

@@ -51,6 +51,7 @@ def lib():
             "oq_selftest_bounded_wait": (i, [vp]),
             "oq_debug_select_rq_kernel": (i, [i]),
             "oq_rq_plan": (i, [vp, vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(sz)]),
+            "oq_rotate_quantize_act_levels": (i, [vp, i, i, i, vp, vp, vp, i, vp, vp, vp, vp]),
             "oq_decode_levels": (i, [vp, i, i, vp, vp, i, vp]),
             "oq_qlinear_levels": (i, [vp, i, vp, i, vp, vp, i, vp, i, vp, i, i, vp]),
             "oq_adaln_packed_bytes": (i, [i, i, C.POINTER(sz), C.POINTER(sz)]),
@@ -233,6 +234,21 @@ def oq_rq_plan(rot, cb):
 
 def oq_debug_select_rq_kernel(which):
     _check(lib().oq_debug_select_rq_kernel(int(which)))
+
+
+def oq_rotate_quantize_act_levels(X, rot, cb_a, out=None, out_norm=None, want_idx=False, dbg_rotated=None):
+    """6-bit activations: X CUDA bf16 [N, d] -> (levels bf16 [N, d], norm fp32 [N], idx uint8 [N, d] or None)."""
+    import torch
+    n, d = X.shape
+    if out is None:
+        out = torch.empty((n, d), dtype=torch.bfloat16, device=X.device)
+    if out_norm is None:
+        out_norm = torch.empty(n, dtype=torch.float32, device=X.device)
+    idx = torch.empty((n, d), dtype=torch.uint8, device=X.device) if want_idx else None
+    _check(lib().oq_rotate_quantize_act_levels(_ptr(X), n, d, X.stride(0) if n > 1 else d, rot.handle, cb_a.handle,
+                                               _ptr(out), out.stride(0) if n > 1 else d, _ptr(out_norm), _ptr(idx),
+                                               _ptr(dbg_rotated), _stream()))
+    return out, out_norm, idx
 
 
 def oq_decode_levels(idx, rows, dim, cb, out=None):

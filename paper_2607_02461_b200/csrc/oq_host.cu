@@ -178,8 +178,11 @@ CodebookParams codebook_params(const oq_codebook* cb) {
   CodebookParams p;
   const int L = 1 << cb->bits, M = L / 2;
   for (int j = 0; j < 8; ++j) p.pos_bound[j] = std::numeric_limits<float>::infinity();
-  for (int j = 1; j < M; ++j) p.pos_bound[j - 1] = cb->boundaries_f32[M - 1 + j];
-  for (int j = 0; j < 16; ++j) p.level_bf16[j] = j < L ? cb->centroids_bf16[j] : 0;
+  for (int j = 0; j < 16; ++j) p.level_bf16[j] = 0;
+  if (cb->bits <= 4) {      // (larger codebooks use WideTables)
+    for (int j = 1; j < M; ++j) p.pos_bound[j - 1] = cb->boundaries_f32[M - 1 + j];
+    for (int j = 0; j < L; ++j) p.level_bf16[j] = cb->centroids_bf16[j];
+  }
   p.bits = cb->bits;
   return p;
 }
@@ -196,6 +199,23 @@ int* device_status_word() {
     g_status_word[dev] = p;
   }
   return g_status_word[dev];
+}
+
+int ensure_wide_tables(const oq_codebook* cb) {
+  if (!cb->wide_ok) return fail(OQ_ERR_UNSUPPORTED, "this codebook has no grid tables (6 bits only)");
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (cb->d_wide && cb->wide_device == dev) return OQ_OK;
+  if (cb->d_wide) return fail(OQ_ERR_INVALID_ARG, "codebook handle was first used on another device");
+  WideTables* d = nullptr;
+  e = cudaMalloc(&d, sizeof(WideTables));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(codebook tables)");
+  e = cudaMemcpy(d, &cb->wide, sizeof(WideTables), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(codebook tables)");
+  cb->d_wide = d;
+  cb->wide_device = dev;
+  return OQ_OK;
 }
 
 int ensure_device_tables(const oq_rpbh* rc) {
@@ -246,14 +266,14 @@ int oq_build_codebook(int dim, int bits, oq_codebook** out) {
   if (!out) return fail(OQ_ERR_INVALID_ARG, "oq_build_codebook: out is NULL");
   *out = nullptr;
   if (dim < 16) return fail(OQ_ERR_UNSUPPORTED, "oq_build_codebook: dim must be >= 16");
-  if (bits < 1 || bits > 4) return fail(OQ_ERR_UNSUPPORTED, "oq_build_codebook: bits must be in 1..4");
+  if (bits < 1 || (bits > 4 && bits != 6)) return fail(OQ_ERR_UNSUPPORTED, "oq_build_codebook: bits must be 1..4 or 6");
   const int L = 1 << bits, M = L / 2;
   const double sigma = 1.0 / std::sqrt((double)dim);
   std::vector<double> c(M), edge(M + 1);
   for (int j = 0; j < M; ++j) c[j] = std::fmin(3.0 * sigma, 1.0) * (2 * j + 1) / (2.0 * M);
   // Plain Lloyd iteration on the positive half (the density is even).  It contracts linearly (ratio
   // about 0.965 at 4 bits), so it runs until the step is at rounding level, with an iteration cap.
-  for (int it = 0; it < 20000; ++it) {
+  for (int it = 0; it < (bits > 4 ? 200000 : 20000); ++it) {
     edge[0] = 0.0;
     for (int j = 1; j < M; ++j) edge[j] = 0.5 * (c[j - 1] + c[j]);
     edge[M] = 1.0;
@@ -281,7 +301,28 @@ int oq_build_codebook(int dim, int bits, oq_codebook** out) {
   cb->centroids_bf16.resize(L);
   for (int j = 0; j < L - 1; ++j) cb->boundaries_f32[j] = (float)cb->boundaries[j];
   for (int j = 0; j < L; ++j) cb->centroids_bf16[j] = f32_to_bf16_rne((float)cb->centroids[j]);
-  if (M > 1) cb->poly = build_quant_poly(&cb->boundaries[M], M - 1);
+  if (M > 1 && bits <= 4) cb->poly = build_quant_poly(&cb->boundaries[M], M - 1);
+  if (bits == 6) {
+    WideTables& w = cb->wide;
+    const float gs = (float)(256.0 / (1.01 * cb->boundaries[L - 2]));
+    w.grid_scale = gs;
+    w.pad[0] = w.pad[1] = w.pad[2] = 0.f;
+    for (int j = 0; j < 32; ++j) {
+      w.bound_scaled[j] = j < M - 1 ? cb->boundaries_f32[M + j] * gs : std::numeric_limits<float>::infinity();
+      w.level_bf16[j] = cb->centroids_bf16[M + j];
+    }
+    bool ok = true;
+    for (int g = 0; g < 256; ++g) {
+      int below = 0, inside = 0;
+      for (int j = 0; j < M - 1; ++j) {
+        if (w.bound_scaled[j] <= (float)g) ++below;
+        else if (w.bound_scaled[j] < (float)(g + 1)) ++inside;
+      }
+      if (inside > 1) ok = false;
+      w.cell[g] = (uint8_t)below;
+    }
+    cb->wide_ok = ok ? 1 : 0;
+  }
   *out = cb;
   return OQ_OK;
 }
@@ -308,7 +349,10 @@ int oq_codebook_level_poly(const oq_codebook* cb, float* coef, float* clamp, flo
 }
 int oq_codebook_dim(const oq_codebook* cb) { return cb ? cb->dim : 0; }
 int oq_codebook_bits(const oq_codebook* cb) { return cb ? cb->bits : 0; }
-void oq_codebook_destroy(oq_codebook* cb) { delete cb; }
+void oq_codebook_destroy(oq_codebook* cb) {
+  if (cb && cb->d_wide) cudaFree(cb->d_wide);
+  delete cb;
+}
 
 int oq_make_rpbh(int dim, int block, uint64_t seed, oq_rpbh** out) {
   if (!out) return fail(OQ_ERR_INVALID_ARG, "oq_make_rpbh: out is NULL");

@@ -22,8 +22,24 @@ struct QuantPoly {
   float mid = 0.f;         // integer constant term
 };
 
+// Tables of a codebook with 64 levels (6 bits), whose level search runs on a uniform grid of the normalised
+// magnitude instead of a polynomial: u = |t| * grid_scale falls into cell g = min(int(u), 255); cell[g] positive
+// boundaries lie at or below the cell's lower edge and at most one lies inside it, so the magnitude rank is
+// cell[g] + (u > bound_scaled[cell[g]]).  Device layout (16-byte aligned, 464 bytes).
+struct WideTables {
+  float bound_scaled[32];    // positive boundaries times grid_scale, ascending; unused entries +inf
+  uint16_t level_bf16[32];   // positive levels, ascending
+  uint8_t cell[256];
+  float grid_scale;          // 256 / (1.01 * largest boundary)
+  float pad[3];
+};
+
 struct oq_codebook {
   int dim = 0, bits = 0;
+  int wide_ok = 0;                   // 6 bits: the grid tables below are valid
+  WideTables wide;
+  mutable WideTables* d_wide = nullptr;   // device copy, created on first GPU use
+  mutable int wide_device = -1;
   QuantPoly poly;
   std::vector<double> centroids;     // 2^bits ascending
   std::vector<double> boundaries;    // 2^bits - 1 midpoints
@@ -51,6 +67,7 @@ namespace oq {
 int fail(int code, const std::string& msg);   // records the message, returns code
 int cuda_fail(cudaError_t e, const char* what);
 int ensure_device_tables(const oq_rpbh* r);   // uploads d_gather on first use
+int ensure_wide_tables(const oq_codebook* cb); // uploads the grid tables of a 6-bit codebook on first use
 
 // Values a kernel needs from a codebook, passed by value as a launch parameter.
 struct CodebookParams {

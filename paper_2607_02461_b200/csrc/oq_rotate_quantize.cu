@@ -199,7 +199,8 @@ struct TcPlan {
   double fill;      // used rows of the operand tiles / all rows
 };
 static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
-  if (block < 64 || block > 4096 || (block & (block - 1)) || !cb->poly.ok) return false;
+  if (block < 64 || block > 4096 || (block & (block - 1))) return false;
+  if (cb->bits == 6 ? !cb->wide_ok : !cb->poly.ok) return false;
   const size_t kMaxSmem = 227 * 1024;
   const int kblocks = dim / 128;
   // blocks above 256: a row's token must be the same in every tile of a group, i.e. th * 2^stages divides 64
@@ -211,7 +212,8 @@ static bool plan_tc(int dim, int block, const oq_codebook* cb, TcPlan* plan) {
     const int pairs = th * kblocks;
     if (pairs > rqtc::MAX_PAIRS) continue;
     // + partial sums, barriers, counters
-    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)rqtc::ROWBUFS * th * rqtc::row_pitch_bytes(dim) + 2 * 16 * 16 * 4 + 256;
+    const size_t base = 1024 + rqtc::OFF_ROWS + (size_t)rqtc::ROWBUFS * th * rqtc::row_pitch_bytes(dim) + 2 * 16 * 16 * 4 + 256 +
+                        (cb->bits == 6 ? 512 : 0);    // (grid tables of a 64-level codebook)
     if (base > kMaxSmem) continue;
     const size_t with_tab = base + (size_t)kblocks * 4 * (rqtc::TAB_PITCH + rqtc::MSK_PITCH);
     const size_t with_tab16 = base + (size_t)kblocks * 4 * rqtc::MSK_PITCH;   // byte offsets fit 16 bits: dim < 32768
@@ -273,6 +275,7 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
     prm.ths = tp.ths; prm.pairs = tp.pairs; prm.ntiles = tp.ntiles;
     prm.bf16_norm = kBf16Norm ? 1 : 0;
     prm.stages = tp.stages;
+    prm.wide = nullptr; prm.out_levels = nullptr; prm.ld_levels = 0; prm.out_idx8 = nullptr; prm.grid_scale = 0.f;
     prm.status = status;
     int grid = sms < prm.groups ? sms : prm.groups;
     if (cb->bits == 4) e = launch_tc_block<4>(rot->block, tp.tab, grid, tp.smem, st, prm);
@@ -318,6 +321,58 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
   return OQ_OK;
 }
 
+// 64-level activation codebook: the levels themselves are the output (bf16 matrix), the operand of oq_qlinear_levels.
+int rotate_quantize_levels_launch(const void* X, int rows, int dim, int ld, const oq_rpbh* rot, const oq_codebook* cb,
+                                  void* out_levels, int ld_levels, float* out_norm, void* out_idx8, float* dbg, int* status,
+                                  void* stream) {
+  const char* fn = "oq_rotate_quantize_act_levels";
+  if (!rot || !cb) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": NULL handle");
+  if (rows < 0 || dim <= 0) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": bad sizes");
+  if (rot->dim != dim || cb->dim != dim)
+    return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": dim differs from the rotation's or the codebook's");
+  if (dim % 128) return fail(OQ_ERR_UNSUPPORTED, std::string(fn) + ": dim must be a multiple of 128");
+  if (cb->bits != 6) return fail(OQ_ERR_UNSUPPORTED, std::string(fn) + ": the codebook must have 6 bits");
+  TcPlan tp;
+  if (!plan_tc(dim, rot->block, cb, &tp))
+    return fail(OQ_ERR_UNSUPPORTED, std::string(fn) + ": block must be 64..4096 and the rows must fit the tensor-core kernel");
+  if (rows == 0) return OQ_OK;
+  if (!X || !out_levels || !out_norm) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": NULL buffer");
+  if (ld < dim || ld_levels < dim) return fail(OQ_ERR_INVALID_ARG, std::string(fn) + ": leading dimension smaller than dim");
+  if (ld % 8 || ld_levels % 8 || !aligned16(X) || !aligned16(out_levels) || (out_idx8 && !aligned16(out_idx8)))
+    return fail(OQ_ERR_ALIGNMENT, std::string(fn) + ": pointers must be 16-byte aligned and leading dimensions multiples of 8");
+  int rc = ensure_device_tables(rot);
+  if (rc != OQ_OK) return rc;
+  rc = ensure_wide_tables(cb);
+  if (rc != OQ_OK) return rc;
+  if (!status) status = device_status_word();
+  if (!status) return fail(OQ_ERR_CUDA, std::string(fn) + ": cannot allocate the device status word");
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  RqTcParams prm;
+  prm.X = reinterpret_cast<const unsigned char*>(X);
+  prm.rows = rows; prm.dim = dim; prm.ldx = ld;
+  prm.offset = rot->d_offset; prm.posmask = rot->d_posmask;
+  prm.out_idx = nullptr; prm.pitch_words = 0;
+  prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
+  const int T = 2 << tp.ths;
+  prm.groups = (rows + T - 1) / T;
+  prm.ths = tp.ths; prm.pairs = tp.pairs; prm.ntiles = tp.ntiles;
+  prm.bf16_norm = 0;
+  prm.stages = tp.stages;
+  prm.wide = cb->d_wide;
+  prm.out_levels = reinterpret_cast<__nv_bfloat16*>(out_levels);
+  prm.ld_levels = ld_levels;
+  prm.out_idx8 = reinterpret_cast<uint8_t*>(out_idx8);
+  prm.grid_scale = cb->wide.grid_scale;
+  prm.status = status;
+  const int grid = sms < prm.groups ? sms : prm.groups;
+  e = launch_tc_block<6>(rot->block, tp.tab, grid, tp.smem, reinterpret_cast<cudaStream_t>(stream), prm);
+  if (e != cudaSuccess) return cuda_fail(e, fn);
+  return OQ_OK;
+}
+
 int rotate_quantize_act_launch(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
                                const oq_codebook* cb_a, void* Xq_idx, float* Xq_norm, float* dbg_rotated, int* status,
                                void* stream) {
@@ -336,6 +391,13 @@ int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, c
                            void* stream) {
   return rotate_quantize_act_launch(X_bf16, n_tokens, dim, ldx, rot, cb_a, Xq_idx, Xq_norm, dbg_rotated, nullptr,
                                     stream);
+}
+
+int oq_rotate_quantize_act_levels(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
+                                  const oq_codebook* cb_a, void* Xd_bf16, int ldxd, float* Xq_norm, void* idx_u8,
+                                  float* dbg_rotated, void* stream) {
+  return rotate_quantize_levels_launch(X_bf16, n_tokens, dim, ldx, rot, cb_a, Xd_bf16, ldxd, Xq_norm, idx_u8, dbg_rotated,
+                                       nullptr, stream);
 }
 
 int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows_per_group, int* tiles_per_group,

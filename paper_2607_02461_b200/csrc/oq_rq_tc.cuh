@@ -60,6 +60,13 @@ struct RqTcParams {
   int ntiles;               // 2 (P <= 128) or 3
   int bf16_norm;            // 1: norms stored as bf16 (weights), 0: fp32 (activations)
   int stages;               // BLK = 512 only: the Hadamard block is 128 << stages (2 .. 5), th << stages <= 64
+  // BITS = 6 (64 levels): the output is the matrix of bf16 levels C[idx] (the operand form of oq_qlinear_levels),
+  // found with the grid tables of WideTables; out_idx is not written
+  const WideTables* wide;   // device
+  __nv_bfloat16* out_levels;
+  int ld_levels;
+  uint8_t* out_idx8;        // optional [rows][dim] level indices 0..63 (tests), or NULL
+  float grid_scale;
   int* status;
 };
 
@@ -85,6 +92,7 @@ enum { WAIT_ROWS = 11, WAIT_AFULL = 12, WAIT_ACC = 13, WAIT_DRAIN = 14, WAIT_AFR
 __host__ __device__ constexpr uint32_t row_pitch_bytes(int dim) { return 2u * (uint32_t)dim + 16u; }
 }  // namespace rqtc
 
+// BITS: 2, 3, 4 (packed indices out, polynomial level search) or 6 (bf16 levels out, grid level search).
 // TAB: where the gather tables live.  0: global memory (read-only path); 1: both copied to shared memory (32-bit
 // offsets, masks); 2: offsets copied to shared memory as 16-bit values, masks stay in global memory.
 // BLK: the Hadamard block, 64, 128 or 256 (256: one butterfly stage across two tile rows after the tensor-core product);
@@ -111,6 +119,8 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
   // [0..2]: gather warps that no longer need row buffer b (never reset; the warp that brings one to a multiple of
   // 8 requests the next copy into it); [3..5]: copies requested per buffer
   unsigned int* s_cnt = reinterpret_cast<unsigned int*>(tmem_slot + 2);
+  // BITS = 6: copy of the grid tables (16-byte aligned: every region above is a multiple of 16 bytes, 144 up to here)
+  const WideTables* s_wide = reinterpret_cast<const WideTables*>(s_cnt + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rows_full0 = smem_u32(bars);          // [3] bulk copies of a half group have landed in buffer b
@@ -188,6 +198,11 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     *reinterpret_cast<uint4*>(smem + OFF_H + (k0 >> 6) * ATOM + n * 128 + ((chunk ^ (n & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
   }
   for (int i = tid; i < 2 * COMPUTE_WARPS * 16; i += THREADS) s_part[i] = 0.f;
+  if constexpr (BITS == 6) {
+    uint32_t* dst = reinterpret_cast<uint32_t*>(s_cnt + 8);
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(p.wide);
+    for (int i = tid; i < (int)(sizeof(WideTables) / 4); i += THREADS) dst[i] = __ldg(src + i);
+  }
   if (TAB == 1) {
     // 16 bytes per thread and load: one or two loads per thread, all in flight together
     const uint4* src = reinterpret_cast<const uint4*>(p.offset);
@@ -362,7 +377,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
     const int tl = row_token(r);
     // lane bits that number the token (the other bits run over the blocks of that token)
     const int tok_bits = BLK == 512 ? (((th - 1) << lg_lo) & 31) : th - 1;
-    const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
+    const Poly2<BITS == 6 ? 1 : (1 << (BITS - 1)) - 1> poly(p.poly);     // (unused with 6 bits)
     const float blk_f = BLK == 512 ? (float)(H << p.stages) : (float)BLK;      // coordinates per Hadamard block
     const float inv_sqrt_h = rsqrtf(blk_f);
     constexpr float mma_h = BLK < H ? (float)BLK : (float)H;   // the tensor-core product multiplies squared norms by this
@@ -430,8 +445,9 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
       }
       const float s0 = __shfl_sync(0xffffffffu, nrm, tl), s1 = __shfl_sync(0xffffffffu, nrm, 8 + tl);
       // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
-      const float kappa0 = 1.0f / (sqrtf(blk_f) * (s0 + 1e-10f) * p.poly.clamp);
-      const float kappa1 = 1.0f / (sqrtf(blk_f) * (s1 + 1e-10f) * p.poly.clamp);
+      // (6 bits: |z| * grid_scale / (sqrt(h) (s + eps)), the position on the level-search grid)
+      const float kappa0 = BITS == 6 ? p.grid_scale / (sqrtf(blk_f) * (s0 + 1e-10f)) : 1.0f / (sqrtf(blk_f) * (s0 + 1e-10f) * p.poly.clamp);
+      const float kappa1 = BITS == 6 ? p.grid_scale / (sqrtf(blk_f) * (s1 + 1e-10f)) : 1.0f / (sqrtf(blk_f) * (s1 + 1e-10f) * p.poly.clamp);
       // ---------------- pass 2: level search and packing; pass 1 of the next group, one tile at a time ----------------
       ssq0 = 0.f;
       ssq1 = 0.f;
@@ -477,6 +493,32 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
 #pragma unroll
             for (int e = 0; e < 32; ++e) d[e] = v[e] * inv_sqrt_h;
           }
+          if constexpr (BITS == 6) {
+            // grid level search (see WideTables): magnitude rank, then the bf16 level with the sign of z (z <= 0
+            // counts as negative: the number of boundaries strictly below the value, as in the packed formats)
+            const float kg = half ? kappa1 : kappa0;
+            uint32_t lv[16], ib[8];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float u = fabsf(v[e]) * kg;
+              const int g = min(__float2int_rz(u), 255);
+              const int cand = s_wide->cell[g];
+              const int mag = cand + (u > s_wide->bound_scaled[cand] ? 1 : 0);
+              const uint32_t neg = v[e] > 0.f ? 0u : 1u;
+              const uint32_t bits = (uint32_t)s_wide->level_bf16[mag] | (neg << 15);
+              const uint32_t idx = neg ? (uint32_t)(31 - mag) : (uint32_t)(32 + mag);
+              if (e & 1) lv[e >> 1] |= bits << 16; else lv[e >> 1] = bits;
+              if (e & 3) ib[e >> 2] |= idx << (8 * (e & 3)); else ib[e >> 2] = idx;
+            }
+            uint4* dl = reinterpret_cast<uint4*>(p.out_levels + (size_t)row * p.ld_levels + j * H + kq * 32);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) dl[c] = make_uint4(lv[4 * c], lv[4 * c + 1], lv[4 * c + 2], lv[4 * c + 3]);
+            if (p.out_idx8 != nullptr) {
+              uint4* di = reinterpret_cast<uint4*>(p.out_idx8 + (size_t)row * p.dim + j * H + kq * 32);
+              di[0] = make_uint4(ib[0], ib[1], ib[2], ib[3]);
+              di[1] = make_uint4(ib[4], ib[5], ib[6], ib[7]);
+            }
+          } else {
           uint32_t words[BITS];
           pack32<BITS>(v, half ? kappa1 : kappa0, poly, words);
           uint32_t* dst = p.out_idx + (size_t)row * p.pitch_words + (j * (H / 32) + kq) * BITS;
@@ -485,6 +527,7 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
           else {
 #pragma unroll
             for (int c = 0; c < BITS; ++c) dst[c] = words[c];
+          }
           }
         }
         // the next group's tile i went into the accumulator that this tile's pass 2 freed (3-tile groups) or one

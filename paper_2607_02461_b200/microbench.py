@@ -46,10 +46,15 @@ def time_kernel(fn, iters, warmup=3, flush_mb=256):
 def run_rq(n, d, bits, block, iters):
     rot, cb = B.oq_make_rpbh(d, block, 0), B.oq_build_codebook(d, bits)
     X = gen_x(n, d)
-    idx = torch.empty((n, B.oq_packed_bytes(n, d, bits)[1]), dtype=torch.uint8, device="cuda")
     nrm = torch.empty(n, dtype=torch.float32, device="cuda")
-    med, best = time_kernel(lambda: B.oq_rotate_quantize_act(X, rot, cb, out_idx=idx, out_norm=nrm), iters)
-    nbytes = 2 * n * d + n * d * bits // 8 + 4 * n
+    if bits == 6:      # 64 levels: the output is the bf16 level matrix
+        lev = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+        med, best = time_kernel(lambda: B.oq_rotate_quantize_act_levels(X, rot, cb, out=lev, out_norm=nrm), iters)
+        nbytes = 2 * n * d + 2 * n * d + 4 * n
+    else:
+        idx = torch.empty((n, B.oq_packed_bytes(n, d, bits)[1]), dtype=torch.uint8, device="cuda")
+        med, best = time_kernel(lambda: B.oq_rotate_quantize_act(X, rot, cb, out_idx=idx, out_norm=nrm), iters)
+        nbytes = 2 * n * d + n * d * bits // 8 + 4 * n
     return {"kernel": "rotate_quantize", "tokens": n, "dim": d, "bits": bits, "block": block, "ms_median": med,
             "ms_min": best, "bytes": nbytes, "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
 

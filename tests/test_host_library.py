@@ -163,3 +163,20 @@ def test_rotate_quantize_plan_rejects_mismatched_handles():
     with pytest.raises(B.OqError) as e:
         B.oq_rq_plan(B.oq_make_rpbh(192, 64, 0), B.oq_build_codebook(192, 4))
     assert e.value.code == 2
+
+
+def test_6bit_codebook_matches_the_stored_oracle_codebook():
+    """64 levels (activations of the W4A6 setting): the library's Lloyd iteration against the oracle's centroids stored
+    under tests/golden/, and the bf16 decode table."""
+    import os
+    from oracle import bf16 as obf
+    for d in (3072, 5120):
+        path = os.path.join(os.path.dirname(__file__), "golden", f"lloyd_max_d{d}_b6.txt")
+        cent = np.array([float(x) for x in open(path).read().split("\n") if x and not x.startswith("#")])
+        cb = B.oq_build_codebook(d, 6)
+        assert np.allclose(cb.centroids, cent, rtol=1e-9, atol=0)
+        assert np.array_equal(cb.centroids_bf16_bits, obf.f64_to_bf16_bits(cent))
+        assert cb.boundaries[31] == 0.0 and np.all(np.diff(cb.boundaries) > 0)
+    with pytest.raises(B.OqError) as e:
+        B.oq_build_codebook(1024, 5)
+    assert e.value.code == 2

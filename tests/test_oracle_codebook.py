@@ -134,3 +134,27 @@ def test_decode_tables():
     assert cb.boundaries_f32.dtype == np.float32 and cb.centroids_bf16_bits.dtype == np.uint16
     assert np.abs(cb.centroids_decoded / cb.centroids - 1).max() <= 2.0 ** -8
     assert np.array_equal(cb.centroids_decoded, -cb.centroids_decoded[::-1])
+
+
+@pytest.mark.parametrize("d", [3072, 5120])
+def test_stored_6bit_codebook_satisfies_the_lloyd_max_conditions(d):
+    """The 64-level codebooks under tests/golden/ (minutes of oracle time each, hence stored) are checked against the
+    defining conditions of Eq. 3's codebook with an independent quadrature: every centroid is the conditional mean of
+    f_d (Eq. 2) over its cell, whose edges are the midpoints of neighbouring centroids; the table is antisymmetric."""
+    import os
+    from scipy import integrate
+    path = os.path.join(os.path.dirname(__file__), "golden", f"lloyd_max_d{d}_b6.txt")
+    c = np.array([float(x) for x in open(path).read().split("\n") if x and not x.startswith("#")])
+    assert c.shape == (64,) and np.all(np.diff(c) > 0)
+    assert np.allclose(c, -c[::-1], rtol=1e-12, atol=0)
+    edges = np.concatenate([[-1.0], 0.5 * (c[:-1] + c[1:]), [1.0]])
+    e = 0.5 * (d - 3)
+    sig = d ** -0.5
+
+    def f(t):
+        return np.exp(e * np.log1p(-t * t))
+    for j in range(32, 64):
+        lo, hi = edges[j], min(edges[j + 1], 12 * sig)
+        mass = integrate.quad(f, lo, hi, epsabs=0, epsrel=1e-12)[0]
+        mom = integrate.quad(lambda t: t * f(t), lo, hi, epsabs=0, epsrel=1e-12)[0]
+        assert abs(mom / mass - c[j]) <= 1e-8 * c[-1]
