@@ -4,6 +4,7 @@
     python -m paper_2607_02461_b200.microbench gemm --tokens 4608 --dim 3072 --m 9216 --bits-a 4 --bits-w 4
     python -m paper_2607_02461_b200.microbench sweep [--quick]     # rotate+quantize bandwidth sweep
     python -m paper_2607_02461_b200.microbench adaln --tokens 1 --dim 3072 --m 18432   # AdaLN INT4 projection
+    python -m paper_2607_02461_b200.microbench step --shape wan --bits-a 6             # whole block step, W4A6 or W4A4
 
 Inputs are synthetic and generated on the GPU (normal values, per-token log-uniform scale, 1% of the
 channels multiplied by 30); these runs time the kernels, parity is covered by the tests.
@@ -90,9 +91,44 @@ def run_adaln(n, d, m, iters):
             "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
 
 
+def run_step(shape, ba, bw, iters):
+    """The four linears of one FLUX- or Wan-shaped block back to back on one stream (rotate+quantize, then GEMM, per
+    layer).  6-bit activations use the bf16-levels operand; 4-bit ones the packed operand."""
+    from . import synth
+    tokens, layers = (synth.FLUX_TOKENS, synth.FLUX_LAYERS) if shape == "flux" else (synth.WAN_TOKENS, synth.WAN_LAYERS)
+    L = []
+    for name, d, m in layers:
+        rot = B.oq_make_rpbh(d, 128, 0)
+        cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
+        W = (torch.randn((m, d), device="cuda") * 0.02).to(torch.bfloat16)
+        wq, wr = B.oq_quantize_weights(W, rot, cbw)
+        del W
+        l = dict(d=d, m=m, rot=rot, cba=cba, cbw=cbw, X=gen_x(tokens, d), wq=wq, wr=wr,
+                 xs=torch.empty(tokens, dtype=torch.float32, device="cuda"),
+                 Y=torch.empty((tokens, m), dtype=torch.bfloat16, device="cuda"))
+        if ba == 6:
+            l["lev"] = torch.empty((tokens, d), dtype=torch.bfloat16, device="cuda")
+        else:
+            l["xq"] = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device="cuda")
+        L.append(l)
+
+    def step():
+        for l in L:
+            if ba == 6:
+                B.oq_rotate_quantize_act_levels(l["X"], l["rot"], l["cba"], out=l["lev"], out_norm=l["xs"])
+                B.oq_qlinear_levels(l["lev"], l["xs"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+            else:
+                B.oq_rotate_quantize_act(l["X"], l["rot"], l["cba"], out_idx=l["xq"], out_norm=l["xs"])
+                B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+    med, best = time_kernel(step, iters)
+    fl = sum(2.0 * tokens * l["m"] * l["d"] for l in L)
+    return {"kernel": "block_step", "shape": shape, "tokens": tokens, "bits_a": ba, "bits_w": bw, "ms_median": med,
+            "ms_min": best, "flops": fl, "tflops": fl / med / 1e9, "tflops_best": fl / best / 1e9}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("mode", choices=["rq", "gemm", "sweep", "adaln"])
+    ap.add_argument("mode", choices=["rq", "gemm", "sweep", "adaln", "step"])
     ap.add_argument("--tokens", type=int, default=17776)
     ap.add_argument("--dim", type=int, default=3072)
     ap.add_argument("--m", type=int, default=9216)
@@ -102,6 +138,7 @@ def main(argv=None):
     ap.add_argument("--block", type=int, default=128)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--shape", choices=["flux", "wan"], default="wan")
     ap.add_argument("--levels", action="store_true", help="gemm: activations as bf16 levels (oq_qlinear_levels)")
     ap.add_argument("--kernel", type=int, default=0, help="rotate+quantize kernel: 0 auto, 1 general, 2 registers, 3 tensor cores")
     a = ap.parse_args(argv)
@@ -111,6 +148,8 @@ def main(argv=None):
         print(json.dumps(run_rq(a.tokens, a.dim, a.bits, a.block, a.iters)))
     elif a.mode == "gemm":
         print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters, a.levels)))
+    elif a.mode == "step":
+        print(json.dumps(run_step(a.shape, a.bits_a, a.bits_w, a.iters)))
     elif a.mode == "adaln":
         print(json.dumps(run_adaln(a.tokens, a.dim, a.m, a.iters)))
     else:
