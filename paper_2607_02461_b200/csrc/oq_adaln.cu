@@ -310,11 +310,9 @@ int oq_adaln_linear(const void* X_bf16, int n_tokens, int ldx, const void* Wq, c
   const size_t smem_max = (size_t)((n_tokens < adaln::MAXN ? n_tokens : adaln::MAXN) + 1) * (dim / 2 + 4) * 4 + red_bytes;
   if (smem_max > 227 * 1024) return fail(OQ_ERR_UNSUPPORTED, "oq_adaln_linear: dim too large for the activation staging buffer");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  static bool attr_set = false;
-  if (!attr_set || smem_max > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(adaln::adaln_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (smem_max > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(adaln::adaln_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return cuda_fail(e, "oq_adaln_linear (shared memory attribute)");
-    attr_set = true;
   }
   // one wave: as many CTAs as are resident at once, each with an equal share of the row tiles (a multiple of RT)
   int dev = 0, sms = 0;

@@ -38,6 +38,8 @@
 #pragma once
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "oq_internal.h"
 #include "oq_rq_fast.cuh"
 #include "oq_sm100.cuh"
@@ -497,27 +499,35 @@ __global__ void __launch_bounds__(rqtc::THREADS, 1) rq_tc_kernel(const RqTcParam
             // grid level search (see WideTables): magnitude rank, then the bf16 level with the sign of z (z <= 0
             // counts as negative: the number of boundaries strictly below the value, as in the packed formats)
             const float kg = half ? kappa1 : kappa0;
-            uint32_t lv[16], ib[8];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float u = fabsf(v[e]) * kg;
-              const int g = min(__float2int_rz(u), 255);
-              const int cand = s_wide->cell[g];
-              const int mag = cand + (u > s_wide->bound_scaled[cand] ? 1 : 0);
-              const uint32_t neg = v[e] > 0.f ? 0u : 1u;
-              const uint32_t bits = (uint32_t)s_wide->level_bf16[mag] | (neg << 15);
-              const uint32_t idx = neg ? (uint32_t)(31 - mag) : (uint32_t)(32 + mag);
-              if (e & 1) lv[e >> 1] |= bits << 16; else lv[e >> 1] = bits;
-              if (e & 3) ib[e >> 2] |= idx << (8 * (e & 3)); else ib[e >> 2] = idx;
-            }
             uint4* dl = reinterpret_cast<uint4*>(p.out_levels + (size_t)row * p.ld_levels + j * H + kq * 32);
+            // (the index bytes are a test output: the loop that does not build them is the one that is timed)
+            auto search32 = [&](auto want_idx) {
+              uint32_t lv[16];
+              [[maybe_unused]] uint32_t ib[8];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) dl[c] = make_uint4(lv[4 * c], lv[4 * c + 1], lv[4 * c + 2], lv[4 * c + 3]);
-            if (p.out_idx8 != nullptr) {
-              uint4* di = reinterpret_cast<uint4*>(p.out_idx8 + (size_t)row * p.dim + j * H + kq * 32);
-              di[0] = make_uint4(ib[0], ib[1], ib[2], ib[3]);
-              di[1] = make_uint4(ib[4], ib[5], ib[6], ib[7]);
-            }
+              for (int e = 0; e < 32; ++e) {
+                const float u = fabsf(v[e]) * kg;
+                const int g = min(__float2int_rz(u), 255);
+                const int cand = s_wide->cell[g];
+                const int mag = cand + (u > s_wide->bound_scaled[cand] ? 1 : 0);
+                const uint32_t neg = v[e] > 0.f ? 0u : 1u;
+                const uint32_t bits = (uint32_t)s_wide->level_bf16[mag] | (neg << 15);
+                if (e & 1) lv[e >> 1] |= bits << 16; else lv[e >> 1] = bits;
+                if constexpr (decltype(want_idx)::value) {
+                  const uint32_t idx = neg ? (uint32_t)(31 - mag) : (uint32_t)(32 + mag);
+                  if (e & 3) ib[e >> 2] |= idx << (8 * (e & 3)); else ib[e >> 2] = idx;
+                }
+              }
+#pragma unroll
+              for (int c = 0; c < 4; ++c) dl[c] = make_uint4(lv[4 * c], lv[4 * c + 1], lv[4 * c + 2], lv[4 * c + 3]);
+              if constexpr (decltype(want_idx)::value) {
+                uint4* di = reinterpret_cast<uint4*>(p.out_idx8 + (size_t)row * p.dim + j * H + kq * 32);
+                di[0] = make_uint4(ib[0], ib[1], ib[2], ib[3]);
+                di[1] = make_uint4(ib[4], ib[5], ib[6], ib[7]);
+              }
+            };
+            if (p.out_idx8 != nullptr) search32(std::true_type{});
+            else search32(std::false_type{});
           } else {
           uint32_t words[BITS];
           pack32<BITS>(v, half ? kappa1 : kappa0, poly, words);
