@@ -112,3 +112,38 @@ def test_w4a6_linear_matches_oracle(n, m, d):
     xq4, xs4 = B.oq_rotate_quantize_act(_dev(xb), rot, cba4)
     y4 = B.oq_qlinear(xq4, xs4, cba4, wq, wr, cbw, d, out_dtype=torch.float32).cpu().numpy().astype(np.float64)
     assert np.linalg.norm(g32 - dense) < np.linalg.norm(y4 - dense)
+
+
+def test_full_flux_size_on_sampled_rows_and_outputs():
+    """4608 tokens x 3072 -> 9216 (the FLUX qkv layer) in the launch configuration the block-step benchmark times:
+    sampled token rows against the oracle's quantizer, sampled outputs against its fp64 product."""
+    import torch
+    n, d, m = 4608, 3072, 9216
+    xb, wb = synth.activations(n, d, seed=5300), synth.weights(m, d, seed=5301)
+    cent = golden_centroids(d)
+    bounds = 0.5 * (cent[:-1] + cent[1:])
+    bounds[31] = 0.0
+    rot, cba, cbw = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, 6), B.oq_build_codebook(d, 4)
+    lev, nrm, idx = B.oq_rotate_quantize_act_levels(_dev(xb), rot, cba, want_idx=True)
+    wq, wr = B.oq_quantize_weights(_dev(wb), rot, cbw)
+    y = B.oq_qlinear_levels(lev, nrm, wq, wr, cbw, d, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    rng = np.random.default_rng(7)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 255, 256, n - 257, n - 256, n - 2, n - 1], rng.choice(n, 246, replace=False)]))
+    perm, signs = orp.make_rpbh(d, 128, 0)
+    ref = oq.quantize_rows(xb[rows], 128, perm, signs, bounds)
+    gi = idx.cpu().numpy()[rows].astype(np.int32)
+    ri = ref["idx"].astype(np.int32)
+    diff = np.abs(gi - ri)
+    assert diff.max() <= 1 and (diff != 0).mean() <= 2e-4
+    assert np.all(np.abs(nrm.cpu().numpy()[rows].astype(np.float64) - ref["norm"]) <= 1e-6 * ref["norm"])
+    assert np.array_equal(_bits(lev)[rows], obf.f64_to_bf16_bits(cent)[gi])
+    cols = np.unique(np.concatenate([[0, 255, 256, m - 1], rng.choice(m, 252, replace=False)]))
+    ow = ocb.lloyd_max(d, 4)
+    iw = B.oq_unpack_indices(wq, m, d, 4).cpu().numpy()[cols]
+    r = obf.bf16_bits_to_f64(_bits(wr))[cols]
+    levels_a = obf.bf16_bits_to_f64(obf.f64_to_bf16_bits(cent))
+    exact = oql.qlinear(gi, nrm.cpu().numpy()[rows], levels_a, iw, r, ow.centroids_decoded)
+    got = y.cpu().numpy().astype(np.float64)[np.ix_(rows, cols)]
+    assert np.linalg.norm(got - exact) <= TOL_F32 * np.linalg.norm(exact)
