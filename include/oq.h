@@ -139,7 +139,8 @@ int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens, const oq_
  * `workspace` is a caller-owned device buffer of at least oq_forward_workspace_bytes() bytes (16-byte
  * aligned); it holds X, the packed activations, the norms and Y while the call is in flight.
  * The call returns after enqueueing; synchronise the stream before reading Y_host_bf16.
- * Errors: as the two calls it wraps, OQ_ERR_NOMEM when the workspace is too small. */
+ * Errors: as the two calls it wraps, OQ_ERR_NOMEM when the workspace is too small.  With a 6-bit activation codebook
+ * the two calls are oq_rotate_quantize_act_levels and oq_qlinear_levels (bits_a = 6 in the size query). */
 int oq_forward_workspace_bytes(int n_tokens, int dim, int m, int bits_a, size_t* bytes);
 int oq_linear_forward_host(const void* X_host_bf16, int n_tokens, int dim, const oq_rpbh* rot,
                            const oq_codebook* cb_a, const void* Wq_idx, const void* Wq_norm_bf16, int m,

@@ -147,3 +147,25 @@ def test_full_flux_size_on_sampled_rows_and_outputs():
     exact = oql.qlinear(gi, nrm.cpu().numpy()[rows], levels_a, iw, r, ow.centroids_decoded)
     got = y.cpu().numpy().astype(np.float64)[np.ix_(rows, cols)]
     assert np.linalg.norm(got - exact) <= TOL_F32 * np.linalg.norm(exact)
+
+
+def test_host_buffer_layer_call_with_6bit_activations():
+    """oq_linear_forward_host with a 64-level activation codebook: same bits as the two calls made by hand."""
+    import torch
+    n, m, d = 300, 520, 3072
+    xb, wb = synth.activations(n, d, seed=5400), synth.weights(m, d, seed=5401)
+    rot, cba, cbw = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, 6), B.oq_build_codebook(d, 4)
+    wq, wr = B.oq_quantize_weights(_dev(wb), rot, cbw)
+    lev, nrm, _ = B.oq_rotate_quantize_act_levels(_dev(xb), rot, cba)
+    want = B.oq_qlinear_levels(lev, nrm, wq, wr, cbw, d)
+    Xh = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+    Yh = torch.empty((n, m), dtype=torch.bfloat16).pin_memory()
+    ws = torch.empty(B.oq_forward_workspace_bytes(n, d, m, 6), dtype=torch.uint8, device="cuda")
+    B.oq_linear_forward_host(Xh, rot, cba, wq, wr, cbw, Yh, ws)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.equal(Yh, want.cpu())
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.OqError) as e:
+        B.oq_linear_forward_host(Xh, rot, cba, wq, wr, cbw, Yh, small)
+    assert e.value.code == 6
