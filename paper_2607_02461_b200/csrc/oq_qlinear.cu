@@ -37,6 +37,13 @@ constexpr uint32_t PSTAGE_BYTES = PA_BYTES + PB_BYTES;                 // 64 KB
 constexpr int EPI_THREADS = 128;
 constexpr int PTHREADS = DECODE_THREADS + EPI_THREADS + 64;   // 16 decode warps, 4 epilogue warps, 1 MMA warp, 1 TMA warp
 constexpr size_t PSMEM_BYTES = PSTAGES * PSTAGE_BYTES + 1024 + 256;
+// Activations as bf16 levels: the TMA-fed activation tiles have a ring of their own, one stage deeper than the
+// weights' (their latency is the L2 round trip of a copy that can only be requested once its buffer is free; the
+// decoders hide theirs by holding the next stage's packed words in registers).
+constexpr int DA_STAGES = 4;
+constexpr uint32_t DB_BASE = DA_STAGES * PA_BYTES;                     // weight ring behind the activation ring
+constexpr uint32_t DBAR_OFF = DB_BASE + PSTAGES * PB_BYTES;            // 224 KB
+constexpr size_t DSMEM_BYTES = DBAR_OFF + 1024 + 256;
 }  // namespace pair
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -112,7 +119,7 @@ __device__ __forceinline__ void dense_b_decode_loop(const uint32_t* __restrict__
   const int lane = threadIdx.x & 31;
   const int atom = tid512 >> 8, t2 = tid512 & 255, row = t2 >> 1, half = t2 & 1;
   const int pitch = dim / 32 * BITS;
-  unsigned char* const tile0 = smem + PA_BYTES + (uint32_t)atom * ATOM_BYTES + (uint32_t)row * 128u;
+  unsigned char* const tile0 = smem + DB_BASE + (uint32_t)atom * ATOM_BYTES + (uint32_t)row * 128u;
   const uint32_t rx = (uint32_t)(row & 7) << 4, c0b = (uint32_t)half * 64u;
   uint32_t st = 0, ph = 0;
   bool first_round = true;
@@ -143,7 +150,7 @@ __device__ __forceinline__ void dense_b_decode_loop(const uint32_t* __restrict__
         if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
         __syncwarp();
       }
-      unsigned char* Ss = tile0 + st * PSTAGE_BYTES;
+      unsigned char* Ss = tile0 + st * PB_BYTES;
       uint4 v[4];
       decode32<BITS>(cur, t, v);
 #pragma unroll
@@ -250,22 +257,27 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
   // 1024-byte alignment computed on the shared-window address: the compiler keeps treating the tiles as shared
   // memory (32-bit addresses) instead of falling back to generic-pointer arithmetic
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + PSTAGES * PSTAGE_BYTES);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PSTAGES + 4);
+  constexpr bool DENSE_A = BITS_A == 0;               // activations as bf16 levels, fetched by TMA
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (DENSE_A ? DBAR_OFF : PSTAGES * PSTAGE_BYTES));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * PSTAGES + 4 + 2 * DA_STAGES);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = cluster_ctarank();
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + PSTAGES);
   const uint32_t accfull0 = smem_u32(bars + 2 * PSTAGES), accempty0 = smem_u32(bars + 2 * PSTAGES + 2);
+  // (levels form only) activation ring: bytes landed / stage read by its MMAs
+  const uint32_t afull0 = smem_u32(bars + 2 * PSTAGES + 4), aempty0 = smem_u32(bars + 2 * PSTAGES + 4 + DA_STAGES);
   constexpr int MMA_WARP = (DECODE_THREADS + EPI_THREADS) / 32, TMA_WARP = MMA_WARP + 1;
-  constexpr bool DENSE_A = BITS_A == 0;               // activations as bf16 levels, fetched by TMA
 
   if (tid == 0) {
     for (int s = 0; s < PSTAGES; ++s) {
-      // one arrival per decoding warp of BOTH CTAs (used in CTA 0); with TMA also one per CTA that announces its bytes
-      mbar_init(full0 + 8 * s, 2 * (DECODE_THREADS / 32) + (DENSE_A ? 2 : 0));
+      mbar_init(full0 + 8 * s, 2 * (DECODE_THREADS / 32));   // one arrival per decoding warp of BOTH CTAs (used in CTA 0)
       mbar_init(empty0 + 8 * s, 1);                          // multicast commit
+    }
+    for (int s = 0; s < DA_STAGES; ++s) {
+      mbar_init(afull0 + 8 * s, 2);                          // one arrival per CTA that announces its bytes (used in CTA 0)
+      mbar_init(aempty0 + 8 * s, 1);                         // multicast commit
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(accfull0 + 8 * b, 1);                        // multicast commit
@@ -303,20 +315,23 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
     // ------------------------------- MMA issuer: one thread of CTA 0 -------------------------------
     if (rank == 0 && lane == 0) {
       uint32_t st = 0, ph = 0, lt = 0;
+      uint32_t sa = 0, pha = 0;                      // stage and phase of the activation ring (levels form)
       constexpr uint32_t IDESC2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
         const uint32_t buf = lt & 1;
         if (lt >= 2) mbar_wait_cluster(accempty0 + 8 * buf, ((lt >> 1) - 1) & 1, abort_flag, status, WAIT_ACC_EMPTY);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         for (int kb = 0; kb < kblocks; ++kb) {
+          if (DENSE_A) mbar_wait_cluster(afull0 + 8 * sa, pha, abort_flag, status, WAIT_FULL);
           mbar_wait_cluster(full0 + 8 * st, ph, abort_flag, status, WAIT_FULL);
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = smem_u32(smem + st * PSTAGE_BYTES);
+          const uint32_t a_addr = smem_u32(smem + (DENSE_A ? sa * PA_BYTES : st * PSTAGE_BYTES));
+          const uint32_t b_addr = smem_u32(smem + (DENSE_A ? DB_BASE + st * PB_BYTES : st * PSTAGE_BYTES + PA_BYTES));
 #pragma unroll
           for (int k4 = 0; k4 < PBK / 16; ++k4) {
             // K step k4: swizzle atom k4 / 4, 32 bytes per step inside the atom
             const uint64_t da = smem_desc(a_addr + (k4 >> 2) * ATOM_BYTES) + 2 * (k4 & 3);
-            const uint64_t db = smem_desc(a_addr + PA_BYTES + (k4 >> 2) * ATOM_BYTES) + 2 * (k4 & 3);
+            const uint64_t db = smem_desc(b_addr + (k4 >> 2) * ATOM_BYTES) + 2 * (k4 & 3);
             const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
             asm volatile(
                 "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
@@ -325,6 +340,10 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
           }
           commit_multicast(empty0 + 8 * st);       // both CTAs may refill the stage once these MMAs have read it
           if (++st == PSTAGES) { st = 0; ph ^= 1; }
+          if (DENSE_A) {
+            commit_multicast(aempty0 + 8 * sa);
+            if (++sa == DA_STAGES) { sa = 0; pha ^= 1; }
+          }
         }
         commit_multicast(accfull0 + 8 * buf);      // both CTAs' epilogue warps may read accumulator `buf`
       }
@@ -332,19 +351,19 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
   } else if (warp == TMA_WARP) {
     // ------------------------------- activation tiles by TMA: one thread per CTA -------------------------------
     if (DENSE_A && lane == 0) {
-      const uint32_t full_leader = map_to_cta(full0, 0);
+      const uint32_t full_leader = map_to_cta(afull0, 0);
       uint32_t st = 0, ph = 0;
       bool first_round = true;
       for (int tile = pair_id; tile < ntiles && !*abort_flag; tile += npairs) {
         const int n0 = (tile / tiles_m) * 256 + (int)rank * 128;       // rows past the last token read as zeros
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!first_round) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
+          if (!first_round) mbar_wait(aempty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
           if (*abort_flag) break;
           mbar_arrive_expect_tx_cluster(full_leader + 8 * st, PA_BYTES);
-          const uint32_t dst = smem_u32(smem + st * PSTAGE_BYTES);
+          const uint32_t dst = smem_u32(smem + st * PA_BYTES);
           tma_load_box(dst, &tmap_a, kb * PBK, n0, full_leader + 8 * st);
           tma_load_box(dst + ATOM_BYTES, &tmap_a, kb * PBK + BK, n0, full_leader + 8 * st);
-          if (++st == PSTAGES) { st = 0; ph ^= 1; first_round = false; }
+          if (++st == DA_STAGES) { st = 0; ph ^= 1; first_round = false; }
         }
       }
       // after a wait gave up somewhere, tiles requested above may still be on their way into this CTA's shared memory:
@@ -491,7 +510,8 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
                         const __nv_bfloat16* wn, int m, int dim, const CodebookParams& ca, const CodebookParams& cw,
                         void* Y, int ldy, int* status) {
   auto k = qlinear_pair_kernel<BA, BW, F32>;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pair::PSMEM_BYTES);
+  constexpr size_t smem_bytes = BA == 0 ? pair::DSMEM_BYTES : pair::PSMEM_BYTES;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
   const int ntiles = ((n + 255) / 256) * ((m + 255) / 256);
   // persistent grid: as many pairs as can be resident at once (SM pairs must sit in one cluster-capable group,
@@ -503,7 +523,7 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sms / 2 * 2);
     cfg.blockDim = dim3(pair::PTHREADS);
-    cfg.dynamicSmemBytes = pair::PSMEM_BYTES;
+    cfg.dynamicSmemBytes = smem_bytes;
     int nclusters = 0;
     e = cudaOccupancyMaxActiveClusters(&nclusters, k, &cfg);
     if (e != cudaSuccess) return e;
@@ -512,7 +532,7 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
   int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev] : sms / 2;
   if (pairs > sms / 2) pairs = sms / 2;
   if (pairs > ntiles) pairs = ntiles;
-  return launch_dependent(k, 2 * pairs, pair::PTHREADS, pair::PSMEM_BYTES, st, tmap, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
+  return launch_dependent(k, 2 * pairs, pair::PTHREADS, smem_bytes, st, tmap, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
 }
 
 template <int BA, int BW>
