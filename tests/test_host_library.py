@@ -180,3 +180,33 @@ def test_6bit_codebook_matches_the_stored_oracle_codebook():
     with pytest.raises(B.OqError) as e:
         B.oq_build_codebook(1024, 5)
     assert e.value.code == 2
+
+
+def test_argument_checks_of_the_newer_entry_points_need_no_device():
+    """Validation comes before any CUDA call: these return their error codes on a machine without a GPU."""
+    L = B.lib()
+    rot = B.oq_make_rpbh(3072, 128, 0)
+    cb4, cb6 = B.oq_build_codebook(3072, 4), B.oq_build_codebook(3072, 6)
+    null = ctypes.c_void_p(0)
+    # 6-bit rotate+quantize wants a 6-bit codebook, and matching dims
+    assert L.oq_rotate_quantize_act_levels(null, 4, 3072, 3072, rot.handle, cb4.handle, null, 3072, null, null, null, null) == 2
+    assert L.oq_rotate_quantize_act_levels(null, 4, 1024, 1024, rot.handle, cb6.handle, null, 1024, null, null, null, null) == 1
+    assert L.oq_rotate_quantize_act_levels(null, 0, 3072, 3072, rot.handle, cb6.handle, null, 3072, null, null, null, null) == 0
+    assert L.oq_rotate_quantize_act_levels(null, 4, 3072, 3072, rot.handle, cb6.handle, null, 3072, null, null, null, null) == 1
+    # the packed-index calls refuse a 6-bit codebook
+    assert L.oq_rotate_quantize_act(null, 4, 3072, 3072, rot.handle, cb6.handle, null, null, null, null) == 2
+    with pytest.raises(B.OqError) as e:
+        B.oq_packed_bytes(4, 3072, 6)
+    assert e.value.code == 2
+    # level-matrix GEMM and decode
+    assert L.oq_qlinear_levels(null, 3072, null, 4, null, null, 8, cb6.handle, 3072, null, 8, 0, null) == 2      # weight bits
+    assert L.oq_qlinear_levels(null, 3072, null, 4, null, null, 8, cb4.handle, 3072, null, 8, 0, null) == 1      # NULL buffers
+    assert L.oq_qlinear_levels(null, 3072, null, 0, null, null, 8, cb4.handle, 3072, null, 8, 0, null) == 0      # nothing to do
+    assert L.oq_decode_levels(null, 4, 3072, cb6.handle, null, 3072, null) == 2
+    assert L.oq_decode_levels(null, 4, 3072, None, null, 3072, null) == 1
+    # AdaLN shapes
+    assert L.oq_adaln_linear(null, 1, 128, null, null, 24, 128, null, 24, 0, null) == 2
+    assert L.oq_adaln_linear(null, 1, 128, null, null, 32, 128, null, 32, 0, null) == 1
+    assert L.oq_adaln_quantize_weights(null, 32, 96, 96, null, null, null) == 2
+    assert B.oq_adaln_packed_bytes(32, 128) == (32 * 128 // 2, 2 * 32 * 128 // 64)
+    assert B.oq_forward_workspace_bytes(10, 3072, 16, 6) > B.oq_forward_workspace_bytes(10, 3072, 16, 4)
