@@ -199,3 +199,10 @@ def test_levels_form_is_bit_identical_to_packed_form(n, m, d, bits_a, bits_w):
     B.oq_decode_levels(xq, n, d, cba, out=wide[:, :d])
     got = B.oq_qlinear_levels(wide[:, :d], xs, wq, wr, cbw, d)
     assert torch.equal(got, B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d))
+
+
+@pytest.mark.parametrize("n,m,d,block", [(200, 520, 3072, 1024), (130, 264, 5120, 1024)])
+def test_whole_layer_with_the_papers_default_block(n, m, d, block):
+    """Both operands rotated with the paper's default block (the largest power of two dividing the width): the rotation
+    cancels in the product (Sec. 4.3) whatever the block, and the layer matches the oracle end to end."""
+    run_case(n, m, d, 4, 4, block=block, seed=3)

@@ -253,3 +253,11 @@ def test_results_are_deterministic(kernel):
     a = B.oq_rotate_quantize_act(X, rot, cb)
     b = B.oq_rotate_quantize_act(X, rot, cb)
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("d,block", [(3072, 1024), (12288, 4096), (13824, 512)])
+def test_weight_rows_with_the_papers_default_blocks(d, block):
+    """Offline weight quantization (Algorithm 1, "Offline") with the default block of each width: bf16 row norms."""
+    wb = synth.weights(72, d, seed=2100 + block)
+    wb[5, :] = 0
+    assert check_rows(wb, block, 3, 4, weights=True) <= 1e-4
