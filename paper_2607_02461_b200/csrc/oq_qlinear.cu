@@ -100,7 +100,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_b
   asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
 }
 // One box of the activation matrix (64 coordinates x 128 rows, 128-byte swizzle) into this CTA's shared memory; the
-// bytes are counted on a barrier of the pair's leading CTA (never a multicast: each CTA fetches its own rows).
+// bytes are counted on a barrier of the pair's leading CTA (each CTA fetches its own rows into its own memory).
 __device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t cluster_bar) {
   asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(cluster_bar), "r"(x), "r"(y) : "memory");
