@@ -390,11 +390,36 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
       for (int c = 0; c < 8; ++c) {
         uint32_t r[32];
         tmem_load32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 256 + c * 32), r);
-        if (trow < n_tokens) {
+        if constexpr (F32_OUT) {
+          if (trow < n_tokens) {
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8) {
+              const int i = i0 + c * 32 + g8 * 8;
+              if (i < m) {
+                const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));
+                const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
+                float y[8];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                  y[2 * jj] = (__uint_as_float(r[g8 * 8 + 2 * jj]) * s) * __uint_as_float(rw[jj] << 16);
+                  y[2 * jj + 1] = (__uint_as_float(r[g8 * 8 + 2 * jj + 1]) * s) * __uint_as_float(rw[jj] & 0xFFFF0000u);
+                }
+                float* dst = reinterpret_cast<float*>(Y) + (size_t)trow * ldy + i;
+                *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
+                *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
+              }
+            }
+          }
+        } else {
+          // bf16: a thread holds 64 contiguous bytes of its row (four 16-byte chunks).  Neighbouring lanes (rows t, t + 1)
+          // swap two chunks each, so that every store instruction writes whole 32-byte sectors: lane pair (2j, 2j + 1)
+          // stores chunks (0, 1) and (2, 3) of row t, then of row t + 1.
+          uint4 pk[4];
 #pragma unroll
           for (int g8 = 0; g8 < 4; ++g8) {
             const int i = i0 + c * 32 + g8 * 8;
-            if (i < m) {
+            pk[g8] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < m) {                               // (uniform over the warp)
               const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));
               const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
               float y[8];
@@ -403,19 +428,31 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
                 y[2 * jj] = (__uint_as_float(r[g8 * 8 + 2 * jj]) * s) * __uint_as_float(rw[jj] << 16);
                 y[2 * jj + 1] = (__uint_as_float(r[g8 * 8 + 2 * jj + 1]) * s) * __uint_as_float(rw[jj] & 0xFFFF0000u);
               }
-              if (F32_OUT) {
-                float* dst = reinterpret_cast<float*>(Y) + (size_t)trow * ldy + i;
-                *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
-                *reinterpret_cast<float4*>(dst + 4) = make_float4(y[4], y[5], y[6], y[7]);
-              } else {
-                __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
-                __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
-                uint4 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(Y) + (size_t)trow * ldy + i) = pk;
-              }
+              __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
+              __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
+              pk[g8].x = *reinterpret_cast<uint32_t*>(&p0); pk[g8].y = *reinterpret_cast<uint32_t*>(&p1);
+              pk[g8].z = *reinterpret_cast<uint32_t*>(&p2); pk[g8].w = *reinterpret_cast<uint32_t*>(&p3);
             }
+          }
+          const bool odd = lane & 1;
+          const uint4 s0 = odd ? pk[0] : pk[1], s1 = odd ? pk[2] : pk[3];
+          uint4 r0, r1;
+          r0.x = __shfl_xor_sync(0xffffffffu, s0.x, 1); r0.y = __shfl_xor_sync(0xffffffffu, s0.y, 1);
+          r0.z = __shfl_xor_sync(0xffffffffu, s0.z, 1); r0.w = __shfl_xor_sync(0xffffffffu, s0.w, 1);
+          r1.x = __shfl_xor_sync(0xffffffffu, s1.x, 1); r1.y = __shfl_xor_sync(0xffffffffu, s1.y, 1);
+          r1.z = __shfl_xor_sync(0xffffffffu, s1.z, 1); r1.w = __shfl_xor_sync(0xffffffffu, s1.w, 1);
+          const int row_a = odd ? trow - 1 : trow, row_b = row_a + 1;
+          const uint4 a0 = odd ? r0 : pk[0], a1 = odd ? r1 : pk[2];
+          const uint4 b0 = odd ? pk[1] : r0, b1 = odd ? pk[3] : r1;
+          const int ca = i0 + c * 32 + (odd ? 8 : 0);
+          __nv_bfloat16* Yb = reinterpret_cast<__nv_bfloat16*>(Y);
+          if (row_a < n_tokens) {
+            if (ca < m) *reinterpret_cast<uint4*>(Yb + (size_t)row_a * ldy + ca) = a0;
+            if (ca + 16 < m) *reinterpret_cast<uint4*>(Yb + (size_t)row_a * ldy + ca + 16) = a1;
+          }
+          if (row_b < n_tokens) {
+            if (ca < m) *reinterpret_cast<uint4*>(Yb + (size_t)row_b * ldy + ca) = b0;
+            if (ca + 16 < m) *reinterpret_cast<uint4*>(Yb + (size_t)row_b * ldy + ca + 16) = b1;
           }
         }
       }
