@@ -146,13 +146,13 @@ __device__ __forceinline__ void dense_b_decode_loop(const uint32_t* __restrict__
     for (int kb = 0; kb < kblocks; ++kb) {
       const Raw<BITS> cur = nxt;
       fetch_next();
+      uint4 v[4];
+      decode32<BITS>(cur, t, v);                       // (registers only: before the stage is known to be free)
       if (!first_round) {
         if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
         __syncwarp();
       }
       unsigned char* Ss = tile0 + st * PB_BYTES;
-      uint4 v[4];
-      decode32<BITS>(cur, t, v);
 #pragma unroll
       for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ((c0b + ((uint32_t)q << 4)) ^ rx)) = v[q];
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
@@ -221,13 +221,16 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
     for (int kb = 0; kb < kblocks; ++kb) {
       const Raw<BITS> c0 = (CONTIG && sub) ? n1r : n0r, c1 = (CONTIG && sub) ? n0r : n1r;
       fetch_next();
+      // the first piece is decoded (registers only) before the stage is known to be free: when the decoders are ahead
+      // of the MMAs, half of the decode arithmetic is off the path from "stage free" to "stage full" (+3-4 %; decoding
+      // both pieces first needs more registers than there are and was slower)
+      uint4 v[4];
+      decode32<BITS>(c0, t, v);
       if (!first_round) {
         if (lane == 0) mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag, status, WAIT_EMPTY);
         __syncwarp();
       }
       unsigned char* Ss = tile0 + st * PSTAGE_BYTES;
-      uint4 v[4];
-      decode32<BITS>(c0, t, v);
 #pragma unroll
       for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(Ss + ((c0b + ((uint32_t)q << 4)) ^ rx)) = v[q];
       decode32<BITS>(c1, t, v);
