@@ -9,7 +9,11 @@ Lloyd-Max level -> pack) followed by the codebook-decode GEMM.  Weights are quan
 
 Prints ONE JSON line (rank 0).  `value` = effective TFLOP/s of the whole step (2*N*m*d summed over the
 layers, divided by the device time of the step, rotate+quantize included), aggregated over ranks
-(token-sharded replicas, no collective).  `--impl reference` times the CPU oracle on a bounded sample.
+(token-sharded replicas, no collective).  At one GPU the same line also carries, measured in the same process
+with the same protocol: `workloads` (the Wan W4A4, FLUX W3A3 and FLUX W2A4 steps), `rq_sweep` (rotate+quantize
+alone on the sweep cells of at least 128 MB) and `sustained` (the GEMMs back to back for two seconds).
+`--gpus N` without a launcher starts N local ranks itself.  `--impl reference` times the CPU oracle on a
+bounded sample.
 """
 import argparse
 import json
@@ -32,6 +36,7 @@ WORKLOADS = {
     "wan_w4a4": (synth.WAN_TOKENS, synth.WAN_LAYERS, 4, 4, 128),
     "single_w4a4": (256, [("linear", 1024, 1024)], 4, 4, 128),
 }
+EXTRA_WORKLOADS = ["wan_w4a4", "flux_w3a3", "flux_w2a4"]      # measured after the headline workload, same process
 CONFIG_INDEX = {"single_w4a4": 0, "flux_w4a4": 1, "flux_w3a3": 1, "flux_w2a4": 2, "wan_w4a4": 3}
 METRIC = "qlinear effective TFLOP/s (whole step: rotate+quantize and codebook GEMM)"
 
@@ -179,52 +184,115 @@ class ClockSampler:
                 "power_w_max": max(self.power) if self.power else None}
 
 
-def run_ours(args):
-    import torch
+# ---- rank plumbing (shared by the GPU arm and by the world-size-2 gloo test) --------------------------------
+def init_ranks(backend, local_device=None):
+    """Joins the process group described by RANK / WORLD_SIZE / LOCAL_RANK / MASTER_* (set by torch.distributed.run).
+    backend: "nccl" on GPUs, "gloo" on CPU.  Returns (rank, world, local_rank); world 1 joins nothing."""
     import torch.distributed as dist
-
-    from paper_2607_02461_b200 import binding as B
-    from paper_2607_02461_b200 import build as oqbuild
-
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        oqbuild.build()          # no-op when liboq.so is newer than its sources
-    if world > 1:
-        dist.barrier()           # the other ranks load the library only after rank 0 has made sure it is built
-    B.lib()
+    if world > 1 and not dist.is_initialized():
+        if backend == "nccl":
+            import torch
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local if local_device is None else local_device))
+        else:
+            dist.init_process_group(backend)
+    return rank, world, local
 
-    tokens, layers, bw, ba, block = WORKLOADS[args.workload]
-    ci = CONFIG_INDEX[args.workload]
-    dev = torch.device("cuda", local)
+
+def rank0_first(rank, world, fn):
+    """Runs fn on rank 0 while the other ranks wait at a barrier (the build step: the other ranks load the library
+    only after rank 0 has made sure that it exists)."""
+    import torch.distributed as dist
+    out = fn() if rank == 0 else None
+    if world > 1:
+        dist.barrier()
+    return out
+
+
+def barrier_all(world, cuda=True):
+    import torch.distributed as dist
+    if world > 1:
+        dist.barrier()
+    if cuda:
+        import torch
+        torch.cuda.synchronize()
+
+
+def max_over_ranks(value, world, device=None):
+    """The slowest rank sets the time: MAX all-reduce of one float64 (control plane only)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(world, flops_per_rank_step, ms_per_step):
+    """Token-sharded replicas, weak scaling: every rank does flops_per_rank_step in the (max over ranks) step time."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+def finish_ranks(world):
+    import torch.distributed as dist
+    if world > 1 and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def spawn_ranks_if_needed(args):
+    """`python bench.py --gpus N` without a launcher: re-run this script under torch.distributed.run with N local ranks
+    (one GPU each), pass its output through and exit with its return code.  Returns False when there is nothing to
+    spawn (one GPU, or already running under a launcher)."""
+    if args.gpus <= 1 or "WORLD_SIZE" in os.environ:
+        return False
+    import socket
+    import subprocess
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
+# ---- one workload on this rank's GPU -------------------------------------------------------------------------
+def prepare_workload(B, workload, dev, rank, host_copies):
+    """Offline part (not timed): codebooks, rotation, weight quantization, device buffers."""
+    import torch
+    tokens, layers, bw, ba, block = WORKLOADS[workload]
+    ci = CONFIG_INDEX[workload]
     to_dev = lambda b: torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
-
-    # ---- offline: codebooks, rotation, weight quantization (not timed) ----
     L = []
     for li, (name, d, m) in enumerate(layers):
         rot = B.oq_make_rpbh(d, block, 0)
         cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
         xb = synth.activations(tokens, d, 1000 + ci + 100 * rank)           # every rank has its own tokens
         wb = synth.weights(m, d, 2000 + 10 * ci + li)
-        Xh = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
-        X = Xh.to(dev)
-        wq, wr = B.oq_quantize_weights(to_dev(wb), rot, cbw)
-        xq = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device=dev)
-        xs = torch.empty(tokens, dtype=torch.float32, device=dev)
-        Y = torch.empty((tokens, m), dtype=torch.bfloat16, device=dev)
-        Yh = torch.empty((tokens, m), dtype=torch.bfloat16).pin_memory()
-        ws = torch.empty(B.oq_forward_workspace_bytes(tokens, d, m, ba), dtype=torch.uint8, device=dev)
-        L.append(dict(name=name, d=d, m=m, rot=rot, cba=cba, cbw=cbw, X=X, Xh=Xh, wq=wq, wr=wr, xq=xq, xs=xs, Y=Y,
-                      Yh=Yh, ws=ws))
+        l = dict(name=name, d=d, m=m, rot=rot, cba=cba, cbw=cbw)
+        if host_copies:
+            l["Xh"] = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
+            l["X"] = l["Xh"].to(dev)
+            l["Yh"] = torch.empty((tokens, m), dtype=torch.bfloat16).pin_memory()
+            l["ws"] = torch.empty(B.oq_forward_workspace_bytes(tokens, d, m, ba), dtype=torch.uint8, device=dev)
+        else:
+            l["X"] = to_dev(xb)
+        l["wq"], l["wr"] = B.oq_quantize_weights(to_dev(wb), rot, cbw)
+        l["xq"] = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device=dev)
+        l["xs"] = torch.empty(tokens, dtype=torch.float32, device=dev)
+        l["Y"] = torch.empty((tokens, m), dtype=torch.bfloat16, device=dev)
+        L.append(l)
         del wb, xb
     torch.cuda.synchronize()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)           # > L2 (126 MB)
+    return L
+
+
+def time_workload(B, L, workload, steps, warmup, flush, world, dev, sampler_factory):
+    """Whole steps bracketed by events (value), then instrumented steps with an event between all kernels (split)."""
+    import torch
+    tokens, layers, bw, ba, block = WORKLOADS[workload]
 
     def step(events=None):
         for l in L:
@@ -237,42 +305,35 @@ def run_ours(args):
         if events is not None:
             e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         flush.zero_()
         step()
-    barrier()
-    sampler = ClockSampler(local, getattr(torch.cuda.get_device_properties(local), "uuid", None)) if rank == 0 else None
+    barrier_all(world)
+    sampler = sampler_factory()
     # The timed region: K steps, one pair of events around each whole step.  Nothing is recorded between the
     # kernels of a step: they are launched with programmatic stream serialisation (a kernel's launch and set-up
     # overlap the tail of the one before it), and an event between two kernels suspends that.
     bracket = []
     t_wall = time.perf_counter()
-    for _ in range(args.steps):
+    for _ in range(steps):
         flush.zero_()                                  # L2 flush between steps (outside the event-timed span)
         a = torch.cuda.Event(enable_timing=True); a.record()
         step()
         b = torch.cuda.Event(enable_timing=True); b.record()
         bracket.append((a, b))
-    barrier()
+    barrier_all(world)
     t_wall = time.perf_counter() - t_wall
     step_ms = [a.elapsed_time(b) for a, b in bracket]
     # The per-kernel split (roofline numbers): the same steps again, right away, with an event between all kernels.
-    inst_steps = max(3, min(args.steps, 20))
+    inst_steps = max(3, min(steps, 20))
     all_events = []
     for _ in range(inst_steps):
         flush.zero_()
         ev = []
         step(ev)
         all_events.append(ev)
-    barrier()
+    barrier_all(world)
     clocks = sampler.stop() if sampler else None
-    status = B.oq_device_status()
-
     inst_ms = float(np.mean([ev[0].elapsed_time(ev[-1]) for ev in all_events]))
     rq_ms = np.zeros(len(L)); gemm_ms = np.zeros(len(L))
     for ev in all_events:
@@ -280,50 +341,152 @@ def run_ours(args):
             rq_ms[i] += ev[2 * i].elapsed_time(ev[2 * i + 1])
             gemm_ms[i] += ev[2 * i + 1].elapsed_time(ev[2 * i + 2])
     rq_ms /= inst_steps; gemm_ms /= inst_steps
-    total_ms = float(np.sum(step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
+    ms_per_step = max_over_ranks(float(np.sum(step_ms)), world, dev) / steps
     flops_step = sum(2 * tokens * l["m"] * l["d"] for l in L)
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    pk = peaks()
+    gemm_tf = flops_step / (float(np.sum(gemm_ms)) * 1e-3) / 1e12
+    rq_b = sum(rq_bytes(tokens, l["d"], ba) for l in L)
+    rq_gbs = rq_b / (float(np.sum(rq_ms)) * 1e-3) / 1e9
+    return {
+        "value": whole_job_tflops(world, flops_step, ms_per_step), "ms_per_step": ms_per_step, "steps": steps,
+        "flops_step": flops_step, "inst_steps": inst_steps, "inst_ms": inst_ms, "wall_s": t_wall, "clocks": clocks,
+        "gemm": {"achieved": gemm_tf, "frac": gemm_tf / pk["bf16_tflops"],
+                 "frac_of_sustained": gemm_tf / pk["bf16_tflops_sustained"], "frac_of_nominal_2250": gemm_tf / 2250.0,
+                 "per_layer_tflops": {l["name"]: 2 * tokens * l["m"] * l["d"] / (gemm_ms[i] * 1e-3) / 1e12
+                                      for i, l in enumerate(L)}},
+        "rq": {"achieved": rq_gbs, "frac": rq_gbs / pk["hbm_gbs"], "frac_of_nominal_8000": rq_gbs / 8000.0,
+               "algorithmic_bytes_per_step": rq_b,
+               "per_layer_gbs": {l["name"]: rq_bytes(tokens, l["d"], ba) / (rq_ms[i] * 1e-3) / 1e9
+                                 for i, l in enumerate(L)}},
+    }
+
+
+def synth_tokens_on_gpu(n, d, seed, dev):
+    """Same recipe as synth.activations, drawn on the GPU (timing-only inputs of the bandwidth sweep)."""
+    import torch
+    g = torch.Generator(device=dev).manual_seed(seed)
+    x = torch.randn((n, d), device=dev, generator=g)
+    x *= torch.exp(torch.empty(n, 1, device=dev).uniform_(-2.3026, 2.3026, generator=g))
+    ch = torch.randperm(d, device=dev, generator=g)[: max(1, round(0.01 * d))]
+    x[:, ch] *= 30.0
+    return x.to(torch.bfloat16)
+
+
+RQ_SWEEP_CELLS = [(17776, 3072), (17776, 12288), (32760, 5120), (32760, 13824), (75600, 3072)]   # footprints >= 128 MB
+
+
+def rq_sweep(B, flush, dev, iters=10):
+    """Rotate+quantize alone on the cells of the bandwidth sweep whose footprint is >= 128 MB (block 128, 3 and 4
+    bits): median of `iters` launches, cold L2 (256 MiB written between launches), CUDA events."""
+    import torch
+    pk = peaks()
+    out = []
+    for n, d in RQ_SWEEP_CELLS:
+        X = synth_tokens_on_gpu(n, d, 7, dev)
+        rot = B.oq_make_rpbh(d, 128, 0)
+        nrm = torch.empty(n, dtype=torch.float32, device=dev)
+        for bits in (3, 4):
+            cb = B.oq_build_codebook(d, bits)
+            idx = torch.empty((n, B.oq_packed_bytes(n, d, bits)[1]), dtype=torch.uint8, device=dev)
+            for _ in range(3):
+                B.oq_rotate_quantize_act(X, rot, cb, out_idx=idx, out_norm=nrm)
+            ts = []
+            for _ in range(iters):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); B.oq_rotate_quantize_act(X, rot, cb, out_idx=idx, out_norm=nrm); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            med = sorted(ts)[len(ts) // 2]
+            gbs = rq_bytes(n, d, bits) / med / 1e6
+            out.append({"tokens": n, "dim": d, "bits": bits, "block": 128, "mb": round(rq_bytes(n, d, bits) / 1e6, 1),
+                        "ms": med, "gbs": gbs, "frac": gbs / pk["hbm_gbs"]})
+            del idx
+        del X
+        torch.cuda.empty_cache()
+    return out
+
+
+def sustained_gemm(B, L, workload, dev, sampler_factory, seconds=2.0):
+    """The workload's GEMMs back to back for >= `seconds` (no flush, no rotate+quantize): the power-capped rate, to be
+    read against the sustained bf16 peak, with the SM clock seen during the loop."""
+    import torch
+    tokens = WORKLOADS[workload][0]
+    flops = sum(2 * tokens * l["m"] * l["d"] for l in L)
+
+    def gemms():
+        for l in L:
+            B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+    gemms(); torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(); gemms(); b.record(); torch.cuda.synchronize()
+    reps = max(10, int(seconds * 1e3 / max(a.elapsed_time(b), 1e-3)) + 1)
+    sampler = sampler_factory()
+    a.record()
+    for _ in range(reps):
+        gemms()
+    b.record(); torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    ms = a.elapsed_time(b)
+    tf = reps * flops / (ms * 1e-3) / 1e12
+    pk = peaks()
+    return {"seconds": ms * 1e-3, "repetitions": reps, "tflops": tf, "frac_of_sustained_peak": tf / pk["bf16_tflops_sustained"],
+            "frac_of_burst_peak": tf / pk["bf16_tflops"], "clocks": clocks}
+
+
+def run_ours(args):
+    import torch
+
+    from paper_2607_02461_b200 import binding as B
+    from paper_2607_02461_b200 import build as oqbuild
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    rank, world, local = init_ranks("nccl")
+    rank0_first(rank, world, oqbuild.build)       # no-op when liboq.so is newer than its sources
+    B.lib()
+    dev = torch.device("cuda", local)
+    uuid = getattr(torch.cuda.get_device_properties(local), "uuid", None)
+    sampler_factory = (lambda: ClockSampler(local, uuid)) if rank == 0 else (lambda: None)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)           # > L2 (126 MB)
+
+    tokens, layers, bw, ba, block = WORKLOADS[args.workload]
+    L = prepare_workload(B, args.workload, dev, rank, host_copies=True)
+    r = time_workload(B, L, args.workload, args.steps, args.warmup, flush, world, dev, sampler_factory)
+    status = B.oq_device_status()
 
     # ---- end to end through the host-buffer entry point: H2D of every layer's tokens and D2H of every Y ----
     # Every layer call (copy in, two kernels, copy out) goes to its own stream, so that the two copy engines
     # and the SMs work on different layers at the same time; the events bracket all of them.
     e2e_steps = max(3, min(args.steps, 10))
     side = [torch.cuda.Stream(device=dev) for _ in L]
-    main = torch.cuda.current_stream()
+    main_stream = torch.cuda.current_stream()
 
     def e2e_step():
         for l, st in zip(L, side):
-            st.wait_stream(main)
+            st.wait_stream(main_stream)
             with torch.cuda.stream(st):
                 B.oq_linear_forward_host(l["Xh"], l["rot"], l["cba"], l["wq"], l["wr"], l["cbw"], l["Yh"], l["ws"])
         for st in side:
-            main.wait_stream(st)
+            main_stream.wait_stream(st)
 
     for _ in range(2):
         e2e_step()
-    barrier()
+    barrier_all(world)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
     e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    barrier_all(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / e2e_steps, world, dev)
     h2d = sum(tokens * l["d"] * 2 for l in L)
     d2h = sum(tokens * l["m"] * 2 for l in L)
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        finish_ranks(world)
         return
     # Context line (a measurement of the box, not a dependency of the path): the library bf16 GEMM of the same
     # shapes on dense operands, timed the same way.
@@ -342,46 +505,71 @@ def run_ours(args):
         mm_ms.append(sorted(ts)[len(ts) // 2])
         del Wd
     pk = peaks()
-    gemm_tf = sum(2 * tokens * l["m"] * l["d"] for l in L) / (float(np.sum(gemm_ms)) * 1e-3) / 1e12
-    rq_b = sum(rq_bytes(tokens, l["d"], ba) for l in L)
-    rq_gbs = rq_b / (float(np.sum(rq_ms)) * 1e-3) / 1e9
-    traffic = None
+    traffic, traffic_source = {}, None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(args.workload, {})
+        tj = json.load(open(tpath))
+        traffic = tj.get(args.workload, {})
+        traffic_source = "profiles/traffic.json: " + str(tj.get("source", "ncu dram bytes per step"))
+    flops_step = r["flops_step"]
+    meets = ("measured burst peak" if r["gemm"]["frac"] >= 0.6 else "none") + \
+            ("; also the nominal 2250 TFLOP/s" if r["gemm"]["frac_of_nominal_2250"] >= 0.6 else "; not the nominal 2250 TFLOP/s")
     out = {
-        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": r["value"], "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "tokens_per_gpu": tokens,
                    "layers": [f"{l['name']} {l['d']}->{l['m']}" for l in L], "bits_w": bw, "bits_a": ba,
                    "rpbh_block": block, "parallelism": f"token-sharded replicas x{world}, no collective",
                    "l2": "256 MiB buffer written between steps, outside the event-timed spans",
-                   "per_kernel_timing": f"{inst_steps} more steps right after the timed region with a CUDA event "
-                                        f"between all kernels ({inst_ms:.4f} ms per step: events between kernels "
+                   "per_kernel_timing": f"{r['inst_steps']} more steps right after the timed region with a CUDA event "
+                                        f"between all kernels ({r['inst_ms']:.4f} ms per step: events between kernels "
                                         f"suspend programmatic dependent launch)"},
-        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel", "achieved": gemm_tf,
-                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemm_tf / pk["bf16_tflops"],
-                     "traffic": (traffic or {}).get("qlinear_bytes_per_step"),
+        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel", "achieved": r["gemm"]["achieved"],
+                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": r["gemm"]["frac"],
+                     "traffic": traffic.get("qlinear_bytes_per_step"), "traffic_source": traffic_source,
                      "peak_source": f"{pk['source']} burst (sustained {pk['bf16_tflops_sustained']})",
-                     "frac_of_nominal_2250": gemm_tf / 2250.0,
-                     "per_layer_tflops": {l["name"]: 2 * tokens * l["m"] * l["d"] / (gemm_ms[i] * 1e-3) / 1e12
-                                          for i, l in enumerate(L)}},
-        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rq_tc_kernel", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
-                                     "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
-                                     "traffic": (traffic or {}).get("rq_bytes_per_step"),
-                                     "algorithmic_bytes_per_step": rq_b, "frac_of_nominal_8000": rq_gbs / 8000.0,
-                                     "per_layer_gbs": {l["name"]: rq_bytes(tokens, l["d"], ba) / (rq_ms[i] * 1e-3) / 1e9
-                                                       for i, l in enumerate(L)}},
-        "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                     "frac_of_nominal_2250": r["gemm"]["frac_of_nominal_2250"],
+                     "target_60pct_met_against": meets,
+                     "per_layer_tflops": r["gemm"]["per_layer_tflops"]},
+        "roofline_rotate_quantize": {"bound": "hbm", "kernel": "rotate+quantize", "achieved": r["rq"]["achieved"],
+                                     "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": r["rq"]["frac"],
+                                     "traffic": traffic.get("rq_bytes_per_step"), "traffic_source": traffic_source,
+                                     "algorithmic_bytes_per_step": r["rq"]["algorithmic_bytes_per_step"],
+                                     "frac_of_nominal_8000": r["rq"]["frac_of_nominal_8000"],
+                                     "per_layer_gbs": r["rq"]["per_layer_gbs"]},
+        "e2e": {"value": whole_job_tflops(world, flops_step, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "context_torch_matmul_bf16": {"unit": "TFLOP/s", "note": "library GEMM on dense bf16 operands of the same shapes",
-                                      "all_layers": sum(2 * tokens * l["m"] * l["d"] for l in L) / (sum(mm_ms) * 1e-3) / 1e12,
+                                      "all_layers": flops_step / (sum(mm_ms) * 1e-3) / 1e12,
                                       "per_layer": {l["name"]: 2 * tokens * l["m"] * l["d"] / (mm_ms[i] * 1e-3) / 1e12
                                                     for i, l in enumerate(L)}},
         "gpu_launches": 2 * len(L) * args.steps,
-        "clocks": clocks, "device_status": status, "wall_s_timed_region": t_wall,
+        "clocks": r["clocks"], "device_status": status, "wall_s_timed_region": r["wall_s"],
     }
+    if world == 1 and not args.no_extras:
+        # The other configurations the targets are stated on, measured in this process with the same protocol
+        # (fewer steps): whole-step TFLOP/s, GEMM and rotate+quantize fractions, clocks per workload.
+        out["sustained"] = sustained_gemm(B, L, args.workload, dev, sampler_factory)
+        del L
+        torch.cuda.empty_cache()
+        extra = {}
+        for wl in EXTRA_WORKLOADS:
+            if wl == args.workload:
+                continue
+            Lw = prepare_workload(B, wl, dev, rank, host_copies=False)
+            rw = time_workload(B, Lw, wl, 5, 3, flush, 1, dev, sampler_factory)
+            extra[wl] = {"value": rw["value"], "ms_per_step": rw["ms_per_step"], "steps": rw["steps"], "warmup": 3,
+                         "gemm_tflops": rw["gemm"]["achieved"], "gemm_frac": rw["gemm"]["frac"],
+                         "gemm_frac_of_sustained": rw["gemm"]["frac_of_sustained"],
+                         "gemm_per_layer_tflops": rw["gemm"]["per_layer_tflops"],
+                         "rq_gbs": rw["rq"]["achieved"], "rq_frac": rw["rq"]["frac"],
+                         "rq_per_layer_gbs": rw["rq"]["per_layer_gbs"], "clocks": rw["clocks"]}
+            del Lw
+            torch.cuda.empty_cache()
+        out["workloads"] = extra
+        out["rq_sweep"] = rq_sweep(B, flush, dev)
+        out["device_status_after_extras"] = B.oq_device_status()
     if world == 1 and not args.no_cpu_baseline:
         stepf, flops, desc = oracle_sample(args.workload)
         stepf()
@@ -393,8 +581,7 @@ def run_ours(args):
                                "cores": min(blas_threads(), len(os.sched_getaffinity(0))), "kind": "oracle",
                                "sample": desc + f", {reps} repetitions"}
     print(json.dumps(out))
-    if world > 1:
-        dist.destroy_process_group()
+    finish_ranks(world)
 
 
 def main():
@@ -405,12 +592,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="flux_w4a4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the other workloads, the rotate+quantize sweep cells and the sustained GEMM loop")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
     else:
+        spawn_ranks_if_needed(args)
         run_ours(args)
 
 

@@ -24,6 +24,8 @@
  *     library (oq_packed_bytes gives the sizes; oq_unpack_indices recovers the logical level indices,
  *     numbered 0 .. 2^bits-1 in ascending order of the level, in rotated-coordinate order).
  *   - There is no CPU fallback: a call that needs the GPU fails with OQ_ERR_CUDA if no device is usable.
+ *   - Threads: handles may be shared between host threads (first-use uploads are serialised inside the library);
+ *     oq_last_error() is per thread; oq_debug_select_rq_kernel is a process-wide test switch and not thread-safe.
  */
 #ifndef OQ_H_
 #define OQ_H_
@@ -102,8 +104,10 @@ int oq_packed_bytes(int rows, int dim, int bits, size_t* idx_bytes, size_t* row_
  *   Xq_idx     dev  packed indices, oq_packed_bytes(n_tokens, dim, bits) bytes, written
  *   Xq_norm    dev  [n_tokens] fp32, s per token, written
  *   dbg_rotated dev [n_tokens][dim] fp32 or NULL; when given, receives x' (test hook; slows the kernel)
- * s is the norm of the raw row (equal to ||Pi x|| because Pi is orthogonal), accumulated in fp32.
- * A zero token gives s = 0 and the lower middle level everywhere.  n_tokens may be 0 (no launch).
+ * s is accumulated in fp32: by the tensor-core kernel (every benchmark width) from the rotated row, as Eq. 8 writes
+ * it; by the register-butterfly and general kernels from the raw row, which is the same number because Pi is
+ * orthogonal.  A coordinate that is exactly on a boundary goes to the lower level (Eq. 3 is silent on ties), so a zero
+ * token gives s = 0 and the lower middle level (2^(bits-1) - 1) everywhere.  n_tokens may be 0 (no launch).
  * Requires dim == rpbh dim == codebook dim, dim % 128 == 0, ldx >= dim, ldx % 8 == 0, 16-byte aligned
  * pointers.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA. */
 int oq_rotate_quantize_act(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
@@ -161,12 +165,13 @@ int oq_linear_forward_host(const void* X_host_bf16, int n_tokens, int dim, const
  * with a message that states both sizes.  `rot` must already have been used by an ordinary GPU call
  * (oq_quantize_weights does that), because creating its device tables allocates; otherwise
  * OQ_ERR_INVALID_ARG.
- * The first call on a device looks up the scratch array's device address and clears its status word with a
- * blocking memset: make that first call before starting any stream capture.
+ * The first call on a device looks up the scratch array's device address (cudaGetSymbolAddress, which may load
+ * the module): make that first call before starting any stream capture.
  * All calls on a device share the one scratch array, which keeps the previous call's contents: two calls
  * whose kernels may overlap on the GPU (different streams) race on it -- serialise them.  Nothing in the
  * scratch needs clearing between calls (every byte that is read was written by the same call); the status
- * word is sticky until oq_device_status reads it. */
+ * word is sticky until oq_device_status reads it, and while it is set every kernel that reports to it gives up
+ * its waits at once, so outputs produced after a time-out are invalid until oq_device_status has been called. */
 int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int dim, int ldx, const oq_rpbh* rot,
                               const oq_codebook* cb_a, const void* Wq_idx, const void* Wq_norm_bf16, int m,
                               const oq_codebook* cb_w, void* Y, int ldy, int y_dtype, void* stream);
@@ -175,9 +180,11 @@ int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int dim, int ldx
  * numbers in rotated-coordinate order. */
 int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream);
 
-/* Synchronises the device and reports (then clears) the device-side status word: 0 when every bounded
- * wait inside the kernels completed, otherwise a code saying which wait gave up.  Returns OQ_OK or
- * OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
+/* Synchronises the device and reports (then clears) the device-side status words (the library's own and the one of
+ * oq_linear_forward_noalloc): 0 when every bounded wait inside the kernels completed, otherwise a code saying which
+ * wait gave up (the first non-zero word; both are cleared).  After a time-out the kernels that report to the same
+ * word cut their waits short until this call has cleared it, so treat every output produced since the previous
+ * clean status as invalid.  Returns OQ_OK or OQ_ERR_DEVICE_TIMEOUT (with *status set), OQ_ERR_CUDA. */
 int oq_device_status(int* status);
 
 /* ---- activations as bf16 levels ("decode once") ----------------------------------------------------- */

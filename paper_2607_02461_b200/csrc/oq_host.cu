@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstring>
 #include <limits>
+#include <mutex>
 #include <new>
 
 #include "oq_internal.h"
@@ -187,15 +188,22 @@ CodebookParams codebook_params(const oq_codebook* cb) {
   return p;
 }
 
+// First-use state (status words, device tables of the handles) is created under one mutex, so that threads making their
+// first call on a device at the same time do not allocate twice or see half-published tables.
+static std::mutex g_first_use_mutex;
 static int* g_status_word[64] = {nullptr};
 
 int* device_status_word() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_first_use_mutex);
   if (!g_status_word[dev]) {
     int* p = nullptr;
     if (cudaMalloc(&p, sizeof(int)) != cudaSuccess) return nullptr;
-    if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) return nullptr;
+    if (cudaMemset(p, 0, sizeof(int)) != cudaSuccess) {
+      cudaFree(p);
+      return nullptr;
+    }
     g_status_word[dev] = p;
   }
   return g_status_word[dev];
@@ -206,50 +214,61 @@ int ensure_wide_tables(const oq_codebook* cb) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  std::lock_guard<std::mutex> lock(g_first_use_mutex);
   if (cb->d_wide && cb->wide_device == dev) return OQ_OK;
   if (cb->d_wide) return fail(OQ_ERR_INVALID_ARG, "codebook handle was first used on another device");
   WideTables* d = nullptr;
   e = cudaMalloc(&d, sizeof(WideTables));
   if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(codebook tables)");
   e = cudaMemcpy(d, &cb->wide, sizeof(WideTables), cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(codebook tables)");
-  cb->d_wide = d;
+  if (e != cudaSuccess) {
+    cudaFree(d);
+    return cuda_fail(e, "cudaMemcpy(codebook tables)");
+  }
   cb->wide_device = dev;
+  cb->d_wide = d;
   return OQ_OK;
 }
 
+// Uploads the four device tables of a rotation.  The handle's pointers are set only after all four exist and hold
+// their data; a failure on the way frees what was allocated and leaves the handle as it was (the next call retries).
 int ensure_device_tables(const oq_rpbh* rc) {
   oq_rpbh* r = const_cast<oq_rpbh*>(rc);
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  std::lock_guard<std::mutex> lock(g_first_use_mutex);
   if (r->d_gather && r->device == dev) return OQ_OK;
   if (r->d_gather) return fail(OQ_ERR_INVALID_ARG, "rpbh handle was first used on another device");
-  std::vector<uint32_t> g(r->dim);
-  for (int k = 0; k < r->dim; ++k) g[k] = (uint32_t)r->perm[k] | (r->signs[k] < 0 ? 0x80000000u : 0u);
-  e = cudaMalloc(&r->d_gather, sizeof(uint32_t) * r->dim);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
-  e = cudaMemcpy(r->d_gather, g.data(), sizeof(uint32_t) * r->dim, cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
-  std::vector<uint32_t> off(r->dim), mask((r->dim + 1) / 2, 0u), pmask((r->dim + 1) / 2, 0u);
+  std::vector<uint32_t> g(r->dim), off(r->dim), mask((r->dim + 1) / 2, 0u), pmask((r->dim + 1) / 2, 0u);
   for (int k = 0; k < r->dim; ++k) {
+    g[k] = (uint32_t)r->perm[k] | (r->signs[k] < 0 ? 0x80000000u : 0u);
     off[k] = 2u * (uint32_t)r->perm[k];
     if (r->signs[k] < 0) {
       mask[r->perm[k] >> 1] |= (r->perm[k] & 1) ? 0x80000000u : 0x00008000u;
       pmask[k >> 1] |= (k & 1) ? 0x80000000u : 0x00008000u;
     }
   }
-  e = cudaMalloc(&r->d_offset, sizeof(uint32_t) * off.size());
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
-  e = cudaMalloc(&r->d_srcmask, sizeof(uint32_t) * mask.size());
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
-  e = cudaMalloc(&r->d_posmask, sizeof(uint32_t) * pmask.size());
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMalloc(rpbh tables)");
-  e = cudaMemcpy(r->d_offset, off.data(), sizeof(uint32_t) * off.size(), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemcpy(r->d_srcmask, mask.data(), sizeof(uint32_t) * mask.size(), cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMemcpy(r->d_posmask, pmask.data(), sizeof(uint32_t) * pmask.size(), cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(rpbh tables)");
+  const std::vector<uint32_t>* host[4] = {&g, &off, &mask, &pmask};
+  uint32_t* dev_tab[4] = {nullptr, nullptr, nullptr, nullptr};
+  const char* what = "cudaMalloc(rpbh tables)";
+  for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+    what = "cudaMalloc(rpbh tables)";
+    e = cudaMalloc(&dev_tab[i], sizeof(uint32_t) * host[i]->size());
+    if (e != cudaSuccess) break;
+    what = "cudaMemcpy(rpbh tables)";
+    e = cudaMemcpy(dev_tab[i], host[i]->data(), sizeof(uint32_t) * host[i]->size(), cudaMemcpyHostToDevice);
+  }
+  if (e != cudaSuccess) {
+    for (int i = 0; i < 4; ++i)
+      if (dev_tab[i]) cudaFree(dev_tab[i]);
+    return cuda_fail(e, what);
+  }
+  r->d_offset = dev_tab[1];
+  r->d_srcmask = dev_tab[2];
+  r->d_posmask = dev_tab[3];
   r->device = dev;
+  r->d_gather = dev_tab[0];      // last: the fast path above tests this pointer
   return OQ_OK;
 }
 
@@ -429,20 +448,23 @@ int oq_device_status(int* status) {
   if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceSynchronize");
   int* w = device_status_word();
   if (!w) return fail(OQ_ERR_CUDA, "oq_device_status: no status word (no usable device?)");
-  e = cudaMemcpy(status, w, sizeof(int), cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
-  if (*status == 0) {
-    // the allocation-free entry point keeps its own status word
-    if (int* w2 = noalloc_status_word()) {
-      e = cudaMemcpy(status, w2, sizeof(int), cudaMemcpyDeviceToHost);
-      if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
-      if (*status != 0) cudaMemset(w2, 0, sizeof(int));
+  // Two words exist: the library's own and the one inside the scratch of the allocation-free entry point.  Both are
+  // read and both are cleared on every call (a word left set would make every later kernel that shares it give up
+  // its waits at once); the first non-zero code is reported.
+  int code[2] = {0, 0};
+  int* word[2] = {w, noalloc_status_word()};
+  for (int i = 0; i < 2; ++i) {
+    if (!word[i]) continue;
+    e = cudaMemcpy(&code[i], word[i], sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy(status)");
+    if (code[i] != 0) {
+      e = cudaMemset(word[i], 0, sizeof(int));
+      if (e != cudaSuccess) return cuda_fail(e, "cudaMemset(status)");
     }
   }
-  if (*status != 0) {
-    cudaMemset(w, 0, sizeof(int));
+  *status = code[0] != 0 ? code[0] : code[1];
+  if (*status != 0)
     return fail(OQ_ERR_DEVICE_TIMEOUT, "a bounded device-side wait gave up; status code " + std::to_string(*status));
-  }
   return OQ_OK;
 }
 

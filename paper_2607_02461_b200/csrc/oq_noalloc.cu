@@ -7,6 +7,7 @@
 // hand-over between the two kernels) and the status word that bounded device-side waits report to.  Here
 // both live in a statically sized device array that is part of the library image, so the call performs no
 // cudaMalloc / cudaFree and uses no allocating library routine.
+#include <mutex>
 #include <string>
 
 #include "oq_internal.h"
@@ -25,6 +26,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
 // Host code cannot use g_noalloc_scratch as an address (on the host the name is only a handle for the
 // symbol); the device address is looked up once per device and cached here.
+std::mutex g_scratch_mutex;
 unsigned char* g_scratch_dev[64] = {nullptr};
 
 int scratch_for_current_device(unsigned char** out) {
@@ -32,13 +34,13 @@ int scratch_for_current_device(unsigned char** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return oq::cuda_fail(e, "cudaGetDevice");
   if (dev < 0 || dev >= 64) return oq::fail(OQ_ERR_UNSUPPORTED, "oq_linear_forward_noalloc: device index above 63");
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
   if (!g_scratch_dev[dev]) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
     if (e != cudaSuccess) return oq::cuda_fail(e, "cudaGetSymbolAddress(scratch)");
-    // the status word must start at zero; the rest is overwritten before it is read
-    e = cudaMemset(p, 0, kNormOffset);
-    if (e != cudaSuccess) return oq::cuda_fail(e, "cudaMemset(scratch status)");
+    // nothing to clear: a static device array starts zeroed when the module is loaded (the status word must start at
+    // zero), and every other byte is written by a call before that call reads it
     g_scratch_dev[dev] = static_cast<unsigned char*>(p);
   }
   *out = g_scratch_dev[dev];
@@ -50,7 +52,9 @@ int scratch_for_current_device(unsigned char** out) {
 namespace oq {
 int* noalloc_status_word() {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || !g_scratch_dev[dev]) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_dev[dev]) return nullptr;
   return reinterpret_cast<int*>(g_scratch_dev[dev]);
 }
 }  // namespace oq

@@ -12,6 +12,7 @@
 // work out of this kernel: the tiles then arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle, no SM
 // instructions), and all 16 decoding warps work on the weights.  Both forms feed the same bf16 values to the same
 // MMAs in the same order: the outputs are bit-identical.
+#include <atomic>
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -526,7 +527,8 @@ cudaError_t make_levels_map(const void* base, int rows, int dim, int ld, CUtenso
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn encode = nullptr;
+  static std::atomic<EncodeFn> encode_cached{nullptr};     // (threads racing here store the same pointer)
+  EncodeFn encode = encode_cached.load(std::memory_order_acquire);
   if (!encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -534,6 +536,7 @@ cudaError_t make_levels_map(const void* base, int rows, int dim, int ld, CUtenso
     if (e != cudaSuccess) return e;
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     encode = reinterpret_cast<EncodeFn>(fn);
+    encode_cached.store(encode, std::memory_order_release);
   }
   const cuuint64_t gdim[2] = {(cuuint64_t)dim, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
@@ -556,10 +559,10 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
   const int ntiles = ((n + 255) / 256) * ((m + 255) / 256);
   // persistent grid: as many pairs as can be resident at once (SM pairs must sit in one cluster-capable group,
   // so this can be fewer than sms / 2)
-  static int max_pairs[64] = {0};
+  static std::atomic<int> max_pairs[64];                    // zero-initialised; threads racing here store the same value
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && max_pairs[dev] == 0) {
+  if (dev >= 0 && dev < 64 && max_pairs[dev].load(std::memory_order_relaxed) == 0) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sms / 2 * 2);
     cfg.blockDim = dim3(pair::PTHREADS);
@@ -567,9 +570,9 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
     int nclusters = 0;
     e = cudaOccupancyMaxActiveClusters(&nclusters, k, &cfg);
     if (e != cudaSuccess) return e;
-    max_pairs[dev] = nclusters > 0 ? nclusters : 1;
+    max_pairs[dev].store(nclusters > 0 ? nclusters : 1, std::memory_order_relaxed);
   }
-  int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev] : sms / 2;
+  int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev].load(std::memory_order_relaxed) : sms / 2;
   if (pairs > sms / 2) pairs = sms / 2;
   if (pairs > ntiles) pairs = ntiles;
   return launch_dependent(k, 2 * pairs, pair::PTHREADS, smem_bytes, st, tmap, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);

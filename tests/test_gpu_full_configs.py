@@ -1,6 +1,7 @@
 """Parity at the benchmark's full sizes (FLUX- and Wan-shaped layers, the rotate+quantize sweep, the W2A4
-drift variant): the GPU processes everything in the launch configuration bench.py times, the oracle checks
-seeded samples of rows and columns that always include both ends and the ragged tile edges."""
+drift variant): the GPU processes everything in the launch configuration bench.py times; the oracle follows 256
+seeded tokens (always both ends and both sides of the ragged tile edges) through every output feature, and a plain
+fp32 product of the library's decoded operands covers every tile of the output."""
 import numpy as np
 import pytest
 
@@ -34,6 +35,8 @@ def sample(n, k, seed, tile=256):
 
 
 def flips_ok(gpu_idx, ref, boundaries):
+    """Checks that every disagreement with the oracle is an adjacent-level flip inside the band; returns the flip rate
+    (exact ties apart) and the positions of all disagreements."""
     gi, ri = gpu_idx.astype(np.int32), ref["idx"].astype(np.int32)
     tmax = np.abs(ref["unit"]).max(axis=1)
     bad = np.argwhere(gi != ri)
@@ -43,10 +46,34 @@ def flips_ok(gpu_idx, ref, boundaries):
         beta = boundaries[min(gi[r, k], ri[r, k])]
         assert abs(ref["unit"][r, k] - beta) <= BAND * tmax[r]
         ties += ref["unit"][r, k] == beta
-    return (len(bad) - ties) / gi.size
+    return (len(bad) - ties) / gi.size, bad
 
 
-def check_layer(n, d, m, ba, bw, xb, wb, block=128, nrows=40, ncols=160, seed=0):
+def whole_output_matches_decoded_product(y, xq, xs, cba, wq, wr, cbw, n, m, d):
+    """Every tile of Y, on the GPU: the library's own decoded level matrices multiplied by a plain fp32 matmul and
+    scaled by both norms.  (Covers the interior tiles that the sampled oracle comparison cannot reach.)"""
+    import torch
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        a = B.oq_decode_levels(xq, n, d, cba).float()
+        w = B.oq_decode_levels(wq, m, d, cbw).float()
+        worst = 0.0
+        for r0 in range(0, n, 4096):
+            ref = (a[r0:r0 + 4096] @ w.T) * xs[r0:r0 + 4096, None] * wr.float()[None, :]
+            got = y[r0:r0 + 4096].float()
+            err = (got - ref).abs()
+            bound = 2.0 ** -8 * ref.abs() + 2e-5 * ref.abs().amax(dim=1, keepdim=True)
+            assert bool((err <= bound).all())
+            worst = max(worst, float(torch.linalg.norm(got - ref) / torch.linalg.norm(ref)))
+        assert worst <= 2e-3
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+
+
+def check_layer(n, d, m, ba, bw, xb, wb, block=128, nrows=256, seed=0):
+    """Whole layer at full size in the launch configuration bench.py times; the oracle follows `nrows` sampled tokens
+    (both ends, both sides of the ragged tile edges) through ALL m output features."""
     import torch
     rot = B.oq_make_rpbh(d, block, 0)
     cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
@@ -57,30 +84,41 @@ def check_layer(n, d, m, ba, bw, xb, wb, block=128, nrows=40, ncols=160, seed=0)
     y = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
     torch.cuda.synchronize()
     assert B.oq_device_status() == 0
-    rows, cols = sample(n, nrows, seed), sample(m, ncols, seed + 1)
+    whole_output_matches_decoded_product(y, xq, xs, cba, wq, wr, cbw, n, m, d)
+    rows = sample(n, nrows, seed)
     ia = B.oq_unpack_indices(xq, n, d, ba)[torch.from_numpy(rows).cuda()].cpu().numpy()
-    iw = B.oq_unpack_indices(wq, m, d, bw)[torch.from_numpy(cols).cuda()].cpu().numpy()
+    iw = B.oq_unpack_indices(wq, m, d, bw).cpu().numpy()
     s = xs.cpu().numpy()[rows]
-    rbits = wr.view(torch.int16).cpu().numpy().view(np.uint16)[cols]
-    got = y[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy().astype(np.float64)
+    rbits = wr.view(torch.int16).cpu().numpy().view(np.uint16)
+    got = y[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64)
     oa, ow = ocb.lloyd_max(d, ba), ocb.lloyd_max(d, bw)
     perm, signs = orp.make_rpbh(d, block, 0)
-    # activation and weight quantization against the oracle on the sampled rows
+    # activation and weight quantization against the oracle: sampled tokens, every weight row
     qa = oq.quantize_rows(xb[rows], block, perm, signs, oa.boundaries)
-    qw = oq.quantize_weight_rows(wb[cols], block, perm, signs, ow.boundaries)
-    fa, fw = flips_ok(ia, qa, oa.boundaries), flips_ok(iw, qw, ow.boundaries)
+    qw = oq.quantize_weight_rows(wb, block, perm, signs, ow.boundaries)
+    (fa, bad_a), (fw, bad_w) = flips_ok(ia, qa, oa.boundaries), flips_ok(iw, qw, ow.boundaries)
     assert fa <= 1e-4 and fw <= 1e-4
     assert np.all(np.abs(s - qa["norm"]) <= 1e-6 * qa["norm"] + 1e-30)
     assert np.abs(rbits.astype(np.int32) - qw["norm_bf16_bits"].astype(np.int32)).max() <= 1
-    # operand-exact and end-to-end products on the sampled block
+    # operand-exact product on the sampled tokens
     ref_op = oql.qlinear(ia, s, oa.centroids_decoded, iw, obf.bf16_bits_to_f64(rbits), ow.centroids_decoded)
-    ref_e2e = oql.qlinear(qa["idx"], qa["norm"].astype(np.float32), oa.centroids_decoded, qw["idx"],
-                          obf.bf16_bits_to_f64(qw["norm_bf16_bits"]), ow.centroids_decoded)
     rel = lambda a, b: np.linalg.norm(a - b) / np.linalg.norm(b)
     assert rel(got, ref_op) <= 2e-3
     slack = 2.0 ** -8 * np.abs(ref_op) + 1e-5 * np.abs(ref_op).max(axis=1, keepdims=True)
     assert np.all(np.abs(got - ref_op) <= slack)
-    assert rel(got, ref_e2e) <= 2e-3 or (fa + fw) > 0      # a band flip at 2-3 bits moves a whole column
+    # end to end: the oracle quantizes the raw inputs itself.  A coordinate within 1e-5 of a boundary may legally go to
+    # either neighbour; the tokens and output features that contain such a coordinate are left out (a single weight
+    # coordinate moves a whole output column by percent at 2-3 bits), everything else must meet the bound.
+    ref_e2e = oql.qlinear(qa["idx"], qa["norm"].astype(np.float32), oa.centroids_decoded, qw["idx"],
+                          obf.bf16_bits_to_f64(qw["norm_bf16_bits"]), ow.centroids_decoded)
+    keep_r = np.setdiff1d(np.arange(len(rows)), np.unique(bad_a[:, 0]) if len(bad_a) else [])
+    keep_c = np.setdiff1d(np.arange(m), np.unique(bad_w[:, 0]) if len(bad_w) else [])
+    dropped = (len(rows) - len(keep_r), m - len(keep_c))
+    assert dropped[0] <= 0.05 * len(rows) and dropped[1] <= 0.05 * m, dropped
+    assert rel(got[np.ix_(keep_r, keep_c)], ref_e2e[np.ix_(keep_r, keep_c)]) <= 2e-3
+    if ba >= 4 and bw >= 4:      # at 4 bits a band flip moves an output by far less than the bound: nothing is left out
+        assert rel(got, ref_e2e) <= 2e-3
+    print(f"flip rates {fa:.2e} / {fw:.2e}; left out of the end-to-end comparison: {dropped[0]} tokens, {dropped[1]} features")
     return fa, fw
 
 
@@ -91,18 +129,19 @@ def test_flux_layers_w4a4(li):
     check_layer(n, d, m, 4, 4, synth.activations(n, d, 1001), synth.weights(m, d, 2010 + li))
 
 
-@pytest.mark.parametrize("ba,bw,li", [(3, 3, 0), (3, 3, 3), (4, 2, 1), (4, 2, 2)])
+@pytest.mark.parametrize("li", range(4))
+@pytest.mark.parametrize("ba,bw", [(3, 3), (4, 2)])
 def test_flux_layers_low_bits(ba, bw, li):
     name, d, m = synth.FLUX_LAYERS[li]
     n = synth.FLUX_TOKENS
     check_layer(n, d, m, ba, bw, synth.activations(n, d, 1001 + (bw == 2)), synth.weights(m, d, 2010 + 10 * (bw == 2) + li))
 
 
-@pytest.mark.parametrize("li", [0, 3])
+@pytest.mark.parametrize("li", range(4))
 def test_wan_layers_w4a4(li):
     name, d, m = synth.WAN_LAYERS[li]
     n = synth.WAN_TOKENS                       # 32760 = 127 * 256 + 248: ragged last token tile
-    check_layer(n, d, m, 4, 4, synth.activations(n, d, 1003), synth.weights(m, d, 2030 + li), nrows=32, ncols=128)
+    check_layer(n, d, m, 4, 4, synth.activations(n, d, 1003), synth.weights(m, d, 2030 + li))
 
 
 def test_w2a4_timestep_drift_reuses_the_fixed_codebook():
@@ -122,7 +161,7 @@ def test_w2a4_timestep_drift_reuses_the_fixed_codebook():
         rows = sample(n, 12, 100 + call)
         ia = B.oq_unpack_indices(xq, n, d, 4)[torch.from_numpy(rows).cuda()].cpu().numpy()
         qa = oq.quantize_rows(xb[rows], 128, perm, signs, oa.boundaries)
-        assert flips_ok(ia, qa, oa.boundaries) <= 1e-4
+        assert flips_ok(ia, qa, oa.boundaries)[0] <= 1e-4
         worst_mse = max(worst_mse, float(d * np.mean((qa["unit"] - oa.centroids[qa["idx"]]) ** 2)))
         assert torch.isfinite(y.float()).all()
     assert B.oq_device_status() == 0
@@ -145,6 +184,6 @@ def test_rotate_quantize_sweep_points(d):
             ia = B.oq_unpack_indices(xq, n, d, bits)[torch.from_numpy(rows).cuda()].cpu().numpy()
             perm, signs = orp.make_rpbh(d, block, 0)
             qa = oq.quantize_rows(xb[rows], block, perm, signs, o.boundaries)
-            assert flips_ok(ia, qa, o.boundaries) <= 1e-4
+            assert flips_ok(ia, qa, o.boundaries)[0] <= 1e-4
             assert np.all(np.abs(xs.cpu().numpy()[rows] - qa["norm"]) <= 1e-6 * qa["norm"])
     assert B.oq_device_status() == 0

@@ -68,7 +68,7 @@ def test_config1_single_linear_w4a4():
     run_case(256, 1024, 1024, 4, 4)
 
 
-@pytest.mark.parametrize("ba,bw", [(3, 3), (4, 2), (4, 3), (2, 2)])
+@pytest.mark.parametrize("ba,bw", [(3, 3), (4, 2), (4, 3), (2, 2), (3, 2), (2, 3), (3, 4), (2, 4)])
 def test_other_bit_widths(ba, bw):
     run_case(200, 512, 1024, ba, bw)
 
