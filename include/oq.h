@@ -250,20 +250,24 @@ int oq_adaln_unpack(const void* Wq, const void* scales, int m, int dim, void* q_
 int oq_selftest_bounded_wait(void* stream);
 
 /* Host-only query (no device needed): which kernel oq_rotate_quantize_act / oq_quantize_weights would launch for
- * this rotation and codebook, and its shape: *kernel = 1 general, 2 register butterflies, 3 tensor cores;
- * *rows_per_group = rows one CTA holds in shared memory at a time (1 for the general kernel);
- * *tiles_per_group = 128-row tensor-core tiles per group (0 for the other kernels); *smem_bytes = dynamic shared
- * memory per CTA.  Any output pointer may be NULL.  Honours oq_debug_select_rq_kernel.  Returns OQ_OK,
- * OQ_ERR_INVALID_ARG (NULL handle, dims differ) or OQ_ERR_UNSUPPORTED (dim not a multiple of 128). */
+ * this rotation and codebook, and its shape: *kernel = 1 general, 2 register butterflies, 3 tensor cores with a
+ * row-per-thread gather, 4 tensor cores with a token-slab gather (only when selected);
+ * *rows_per_group = rows one CTA holds in shared memory at a time (1 for the general kernel; the tokens of a slab for
+ * kernel 4); *tiles_per_group = 128-row tensor-core tiles per group (0 for kernels 1 and 2, 1 for kernel 4);
+ * *smem_bytes = dynamic shared memory per CTA.  Any output pointer may be NULL.  Honours oq_debug_select_rq_kernel.
+ * Returns OQ_OK, OQ_ERR_INVALID_ARG (NULL handle, dims differ) or OQ_ERR_UNSUPPORTED (dim not a multiple of 128). */
 int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows_per_group, int* tiles_per_group,
                size_t* smem_bytes);
 
 /* Test helper: selects the kernel behind oq_rotate_quantize_act / oq_quantize_weights for the following calls of
  * this process: 0 = choose by shape (default), 1 = general kernel (any block size; butterflies in shared memory),
  * 2 = register-butterfly kernel (blocks of 64, 128, 256), 3 = tensor-core kernel (blocks of 64 to 4096; the block
- * Hadamard transform of Eq. 7 as a product with a 128 x 128 matrix of +-1, plus butterfly stages for larger blocks).  A selected kernel that does not
- * support the shape falls back to the general one.  All three compute the same function; the parity tests run
- * each of them.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
+ * Hadamard transform of Eq. 7 as a product with a 128 x 128 matrix of +-1, plus butterfly stages for larger blocks;
+ * every thread gathers the coordinates of one row), 4 = token-slab tensor-core kernel (blocks of 64, 128, 256, rows of
+ * 1024 coordinates and more: the rows of 8, 4 or 2 tokens are transposed so that one shared-memory access moves a
+ * coordinate of all of them, and the row norms come from a Gram product on the tensor cores; never chosen by shape,
+ * it measured slower).  A selected kernel that does not support the shape falls back.  All of them compute the same
+ * function; the parity tests run each of them.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
 int oq_debug_select_rq_kernel(int which);
 
 const char* oq_last_error(void);

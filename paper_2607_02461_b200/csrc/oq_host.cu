@@ -1,5 +1,6 @@
 // Host side of liboq: error reporting, the two offline constructors (Lloyd-Max codebook, RPBH draw),
 // size queries and the device status word.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <limits>
@@ -188,6 +189,32 @@ CodebookParams codebook_params(const oq_codebook* cb) {
   return p;
 }
 
+cudaError_t encode_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                                   const uint32_t* box) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static std::atomic<EncodeFn> cached{nullptr};       // (threads racing here store the same pointer)
+  EncodeFn encode = cached.load(std::memory_order_acquire);
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    encode = reinterpret_cast<EncodeFn>(fn);
+    cached.store(encode, std::memory_order_release);
+  }
+  cuuint64_t gdim[3] = {1, 1, 1}, gstride[2] = {0, 0};
+  cuuint32_t bx[3] = {1, 1, 1}, estride[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) gstride[i] = strides_bytes[i];
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, bx, estride,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 // First-use state (status words, device tables of the handles) is created under one mutex, so that threads making their
 // first call on a device at the same time do not allocate twice or see half-published tables.
 static std::mutex g_first_use_mutex;
@@ -249,10 +276,24 @@ int ensure_device_tables(const oq_rpbh* rc) {
       pmask[k >> 1] |= (k & 1) ? 0x80000000u : 0x00008000u;
     }
   }
-  const std::vector<uint32_t>* host[4] = {&g, &off, &mask, &pmask};
-  uint32_t* dev_tab[4] = {nullptr, nullptr, nullptr, nullptr};
+  // token-slab kernel: where the chunk of every rotated position sits inside a slab buffer
+  std::vector<uint32_t> mm;
+  RqMmShape shape;
+  const int mm_tok = rq_mm_shape(r->dim, &shape) ? shape.tok : 0;
+  if (mm_tok) {
+    mm.resize(r->dim);
+    const int nb = r->dim / 128;
+    for (int j = 0; j < nb; ++j)
+      for (int k = 0; k < 128; ++k)
+        mm[j * 128 + (k % 8) * 16 + k / 8] = rq_mm_chunk_offset(r->perm[j * 128 + k], mm_tok, nb);
+  } else {
+    mm.assign(4, 0u);
+  }
+  const int ntab = 5;
+  const std::vector<uint32_t>* host[ntab] = {&g, &off, &mask, &pmask, &mm};
+  uint32_t* dev_tab[ntab] = {nullptr, nullptr, nullptr, nullptr, nullptr};
   const char* what = "cudaMalloc(rpbh tables)";
-  for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+  for (int i = 0; i < ntab && e == cudaSuccess; ++i) {
     what = "cudaMalloc(rpbh tables)";
     e = cudaMalloc(&dev_tab[i], sizeof(uint32_t) * host[i]->size());
     if (e != cudaSuccess) break;
@@ -260,10 +301,12 @@ int ensure_device_tables(const oq_rpbh* rc) {
     e = cudaMemcpy(dev_tab[i], host[i]->data(), sizeof(uint32_t) * host[i]->size(), cudaMemcpyHostToDevice);
   }
   if (e != cudaSuccess) {
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < ntab; ++i)
       if (dev_tab[i]) cudaFree(dev_tab[i]);
     return cuda_fail(e, what);
   }
+  r->d_mm_table = dev_tab[4];
+  r->mm_tok = mm_tok;
   r->d_offset = dev_tab[1];
   r->d_srcmask = dev_tab[2];
   r->d_posmask = dev_tab[3];
@@ -428,6 +471,7 @@ void oq_rpbh_destroy(oq_rpbh* r) {
   if (r->d_offset) cudaFree(r->d_offset);
   if (r->d_srcmask) cudaFree(r->d_srcmask);
   if (r->d_posmask) cudaFree(r->d_posmask);
+  if (r->d_mm_table) cudaFree(r->d_mm_table);
   delete r;
 }
 

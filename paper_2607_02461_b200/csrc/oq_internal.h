@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of liboq (not installed).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string>
@@ -60,9 +61,63 @@ struct oq_rpbh {
                                  // element moves to a position whose sign is -1
   uint32_t* d_posmask = nullptr; // [dim/2] bf16x2 sign-bit masks indexed by ROTATED position: bit 15 / bit 31 set where
                                  // position 2i / 2i+1 has sign -1
+  uint32_t* d_mm_table = nullptr; // [dim] token-slab kernel: byte offset, inside a slab buffer, of the chunk of rotated
+                                 // position (j, k), stored at j * 128 + (k % 8) * 16 + k / 8; NULL when mm_tok == 0
+  int mm_tok = 0;                // tokens per slab of the token-slab kernel for this width (8, 4, 2), 0: not supported
 };
 
 namespace oq {
+
+// ---- layout of the token-slab rotate+quantize kernel (shared by the kernel, its launcher and the table builder) ----
+// A slab is `tok` consecutive tokens (8, 4 or 2 by row length).  Its rows are transposed into a slab buffer of
+// 16-byte rows: a row holds 8 / tok source coordinates (32 apart) of all tok tokens, the tok values of one
+// coordinate adjacent (a "chunk").  The tensor cores read the buffer as both operands of a Gram product, as an
+// MN-major matrix with the 128-byte swizzle: two halves of 8 * seg_rows rows each (seg_rows a multiple of 16), of which
+// the last 8 * pad_rows rows are unused and stay zero.
+// position of source coordinate cb (0..31) of a window among the window's 32 rows of the slab buffer: the 8 rows
+// that one stmatrix phase writes fall into 8 different 16-byte bank groups
+__host__ __device__ constexpr int rq_mm_window_row(int cb) { return (cb & ~7) | ((cb + 2 * (cb >> 3)) & 7); }
+// Byte offset, inside a slab buffer, of the chunk (tok tokens x 2 bytes) of source coordinate i.
+inline uint32_t rq_mm_chunk_offset(int i, int tok, int nb) {
+  const int hw = 8 / tok;                       // coordinates that share one 16-byte row
+  const int w = i / (32 * hw), r = i % (32 * hw), h = r / 32, cb = r % 32;
+  const int raw = nb * tok, seg_rows = (raw + 15) / 16 * 16;
+  const int lin = w * 32 + rq_mm_window_row(cb);
+  const int row = lin + (lin >= 8 * raw ? 8 * (seg_rows - raw) : 0);
+  return 16u * (uint32_t)row + (uint32_t)(h * 2 * tok);
+}
+struct RqMmShape {
+  int tok, seg_rows, pad_rows, nstages, tab_smem, mask_smem;
+  size_t smem;
+};
+// false: this width does not run on the token-slab kernel.  The largest slab that fits in shared memory beside the
+// Hadamard tile (32 KB) and the operand tile (32 KB); a tile of 128 / tok chunks must not touch more than the two
+// slabs that are resident.
+inline bool rq_mm_shape(int dim, RqMmShape* shape) {
+  if (dim <= 0 || dim % 128) return false;
+  const size_t kMaxSmem = 227 * 1024;
+  const int nb = dim / 128;
+  for (int tok = 8; tok >= 2; tok >>= 1) {
+    const int hw = 8 / tok, bc = 128 / tok;
+    if (dim % (32 * hw)) continue;
+    if (!(nb >= bc - 1 || (bc % nb == 0 && bc / nb <= 2))) continue;
+    const int raw = nb * tok, seg_rows = (raw + 15) / 16 * 16;
+    if (seg_rows > 16383) continue;
+    const size_t slab = 256 * (size_t)seg_rows;
+    // what else goes to shared memory, in order of preference: the sign masks (read once per 8 coordinates), then the
+    // gather table (read once per chunk, in batches); what stays out is read through L1
+    for (int opt = 3; opt >= 0; --opt) {
+      const int mask = (opt == 3 || opt == 2) ? 1 : 0, tab = (opt == 3 || opt == 1) ? 1 : 0;
+      const size_t smem = 1024 + 65536 + 2 * slab + (tab ? 4 * (size_t)dim : 0) + (mask ? 2 * (size_t)dim : 0) + 3072;
+      if (smem <= kMaxSmem) {
+        shape->tok = tok; shape->seg_rows = seg_rows; shape->pad_rows = seg_rows - raw;
+        shape->nstages = 0; shape->tab_smem = tab; shape->mask_smem = mask; shape->smem = smem;
+        return true;
+      }
+    }
+  }
+  return false;
+}
 
 int fail(int code, const std::string& msg);   // records the message, returns code
 int cuda_fail(cudaError_t e, const char* what);
@@ -76,6 +131,11 @@ struct CodebookParams {
   int bits;
 };
 CodebookParams codebook_params(const oq_codebook* cb);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time dependency on the driver library).
+// bf16 elements, no interleave, no swizzle, out-of-bounds elements read as zero.  rank <= 3.
+cudaError_t encode_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                                   const uint32_t* box);
 
 // Device status word (bounded waits report here).
 int* device_status_word();   // device pointer (allocated on first use), or nullptr on failure

@@ -5,6 +5,7 @@
 #include "oq_internal.h"
 #include "oq_packing.cuh"
 #include "oq_rq_fast.cuh"
+#include "oq_rq_mm_params.h"
 #include "oq_rq_tc.cuh"
 
 namespace oq {
@@ -184,9 +185,22 @@ static cudaError_t launch_fast_T(int bits, int grid, const FastPlan& pl, cudaStr
   return cudaErrorInvalidValue;
 }
 
-// Which rotate+quantize kernel to use: 0 = choose by shape, 1 = general, 2 = register butterflies, 3 = tensor
-// cores.  A forced kernel that cannot handle the shape falls back to the general one.
+// Which rotate+quantize kernel to use: 0 = choose by shape (never the token-slab kernel: it measured slower than the
+// row-per-thread one on every benchmark shape), 1 = general, 2 = register butterflies, 3 = tensor cores (row-per-thread
+// gather), 4 = tensor cores (token-slab gather).  A forced kernel that cannot handle the shape falls back.
 static int g_forced_kernel = 0;
+static int g_mm_desc_swap = 0;      // test switch of the token-slab kernel's operand descriptors
+
+// Token-slab kernel: blocks of 64, 128, 256; packed outputs; widths for which rq_mm_shape finds a slab size.
+static bool plan_mm(int dim, int block, const oq_codebook* cb, RqMmShape* shape) {
+  if (block != 64 && block != 128 && block != 256) return false;
+  if (cb->bits < 2 || cb->bits > 4 || !cb->poly.ok) return false;
+  if (!rq_mm_shape(dim, shape)) return false;
+  if (block == 256 && (dim / 128) % 2) return false;
+  return true;
+}
+
+cudaError_t rq_mm_launch(int bits, int tok, int block, int grid, size_t smem, cudaStream_t st, const RqMmParams& prm);   // oq_rq_mm.cu
 
 // Plan of the tensor-core kernel: th tokens per half group (1, 2, 4 or 8), the largest for which the
 // P = th * dim / 128 (token, block) pairs of a half number at most 192 and three half groups of rows fit in
@@ -259,6 +273,27 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
   cudaGetDevice(&dev);
   cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+  RqMmShape ms;
+  if (g_forced_kernel == 4 && plan_mm(dim, rot->block, cb, &ms) && rot->mm_tok == ms.tok) {
+    if (!status) status = device_status_word();
+    if (!status) return fail(OQ_ERR_CUDA, std::string(fn) + ": cannot allocate the device status word");
+    RqMmParams prm;
+    prm.X = reinterpret_cast<const unsigned char*>(X);
+    prm.rows = rows; prm.dim = dim; prm.ldx = ld;
+    prm.table = rot->d_mm_table; prm.srcmask = rot->d_srcmask;
+    prm.out_idx = reinterpret_cast<uint32_t*>(out_idx); prm.pitch_words = pitch_words;
+    prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
+    prm.nslabs = (rows + ms.tok - 1) / ms.tok;
+    prm.nb = dim / 128;
+    prm.seg_rows = ms.seg_rows; prm.pad_rows = ms.pad_rows; prm.nstages = ms.nstages; prm.tab_smem = ms.tab_smem; prm.mask_smem = ms.mask_smem;
+    prm.bf16_norm = kBf16Norm ? 1 : 0;
+    prm.desc_swap = g_mm_desc_swap;
+    prm.status = status;
+    const int grid = sms < prm.nslabs ? sms : prm.nslabs;
+    e = rq_mm_launch(cb->bits, ms.tok, rot->block, grid, ms.smem, st, prm);
+    if (e != cudaSuccess) return cuda_fail(e, fn);
+    return OQ_OK;
+  }
   TcPlan tp;
   const bool tc_ok = plan_tc(dim, rot->block, cb, &tp);
   if ((g_forced_kernel == 0 && tc_ok && tp.fill >= 0.6) || (g_forced_kernel == 3 && tc_ok)) {
@@ -409,8 +444,11 @@ int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows
   size_t smem = (size_t)rot->dim * 5;
   TcPlan tp;
   FastPlan fp;
+  RqMmShape ms;
   const bool tc_ok = plan_tc(rot->dim, rot->block, cb, &tp);
-  if ((g_forced_kernel == 0 && tc_ok && tp.fill >= 0.6) || (g_forced_kernel == 3 && tc_ok)) {
+  if (g_forced_kernel == 4 && plan_mm(rot->dim, rot->block, cb, &ms)) {
+    k = 4; rows = ms.tok; tiles = 1; smem = ms.smem;
+  } else if ((g_forced_kernel == 0 && tc_ok && tp.fill >= 0.6) || (g_forced_kernel == 3 && tc_ok)) {
     k = 3; rows = 2 << tp.ths; tiles = tp.ntiles; smem = tp.smem;
   } else if (g_forced_kernel != 1 && plan_fast(rot->dim, rot->block, cb, &fp)) {
     k = 2; rows = fp.T; smem = fp.smem;
@@ -423,7 +461,11 @@ int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows
 }
 
 int oq_debug_select_rq_kernel(int which) {
-  if (which < 0 || which > 3) return fail(OQ_ERR_INVALID_ARG, "oq_debug_select_rq_kernel: which must be 0..3");
+  if (which >= 100 && which <= 101) {      // 100 / 101: stride fields of the token-slab kernel's descriptors as built / exchanged
+    g_mm_desc_swap = which - 100;
+    return OQ_OK;
+  }
+  if (which < 0 || which > 4) return fail(OQ_ERR_INVALID_ARG, "oq_debug_select_rq_kernel: which must be 0..4");
   g_forced_kernel = which;
   return OQ_OK;
 }

@@ -20,7 +20,7 @@ def _dev(bits_u16):
     return torch.from_numpy(bits_u16.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-AUTO, GENERAL, REGISTERS, TENSOR = 0, 1, 2, 3    # oq_debug_select_rq_kernel
+AUTO, GENERAL, REGISTERS, TENSOR, SLAB = 0, 1, 2, 3, 4    # oq_debug_select_rq_kernel
 
 
 @pytest.fixture(autouse=True)
@@ -83,11 +83,12 @@ def test_activation_rows_match_oracle(d, block, bits):
     assert rate <= 1e-4
 
 
-@pytest.mark.parametrize("kernel", [GENERAL, REGISTERS, TENSOR])
+@pytest.mark.parametrize("kernel", [GENERAL, REGISTERS, TENSOR, SLAB])
 @pytest.mark.parametrize("bits", [4, 3, 2])
-@pytest.mark.parametrize("d,n", [(128, 67), (256, 40), (1024, 67), (3072, 67), (5120, 35), (12288, 21), (13824, 9)])
+@pytest.mark.parametrize("d,n", [(128, 67), (256, 40), (1024, 67), (2048, 35), (3072, 67), (5120, 35), (12288, 21), (13824, 9)])
 def test_every_kernel_matches_oracle_on_blocks_of_128(d, n, bits, kernel):
-    """The three kernels compute the same function; blocks of 128 are the shape all of them support."""
+    """The four kernels compute the same function; blocks of 128 are the shape all of them support (the token-slab
+    kernel from 1024 coordinates per row on; below that the selection falls back)."""
     xb = synth.activations(n, d, seed=1100 + bits)
     assert check_rows(xb, 128, 1, bits, kernel=kernel) <= 1e-4
 
@@ -95,11 +96,12 @@ def test_every_kernel_matches_oracle_on_blocks_of_128(d, n, bits, kernel):
 @pytest.mark.parametrize("bits", [4, 3])
 @pytest.mark.parametrize("block", [64, 256])
 @pytest.mark.parametrize("d,n", [(256, 40), (1024, 67), (3072, 67), (5120, 35), (12288, 21), (13824, 9)])
-def test_tensor_core_kernel_on_blocks_of_64_and_256(d, n, block, bits):
+@pytest.mark.parametrize("kernel", [TENSOR, SLAB])
+def test_tensor_core_kernels_on_blocks_of_64_and_256(d, n, block, bits, kernel):
     """Blocks of 64 are two independent transforms per 128-coordinate tile row (block-diagonal operand); blocks of
     256 add one butterfly stage across the two tile rows of a block."""
     xb = synth.activations(n, d, seed=1300 + bits)
-    assert check_rows(xb, block, 5, bits, kernel=TENSOR) <= 1e-4
+    assert check_rows(xb, block, 5, bits, kernel=kernel) <= 1e-4
 
 
 @pytest.mark.parametrize("bits", [4, 3, 2])
@@ -139,7 +141,7 @@ def test_large_blocks_with_few_rows_match_the_general_kernel(n, d, block):
     assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 2e-4
 
 
-@pytest.mark.parametrize("kernel", [REGISTERS, TENSOR])
+@pytest.mark.parametrize("kernel", [REGISTERS, TENSOR, SLAB])
 def test_kernels_agree_with_each_other_on_many_groups(kernel):
     """More row groups than CTAs (several pipeline rounds per CTA), ragged last group: same packed words and
     norms (to rounding) as the general kernel."""
@@ -162,9 +164,10 @@ def test_kernels_agree_with_each_other_on_many_groups(kernel):
     assert int(diff.max()) <= 1 and float((diff != 0).float().mean()) <= 1e-4
 
 
-@pytest.mark.parametrize("n", [1, 2, 15, 16, 17, 31, 33])
-@pytest.mark.parametrize("d,block", [(3072, 128), (12288, 64), (5120, 256)])
-def test_tensor_core_kernel_with_few_rows_and_padded_rows(n, d, block):
+@pytest.mark.parametrize("kernel", [TENSOR, SLAB])
+@pytest.mark.parametrize("n", [1, 2, 7, 8, 9, 15, 16, 17, 31, 33])
+@pytest.mark.parametrize("d,block", [(3072, 128), (12288, 64), (5120, 256), (13824, 128), (1024, 128)])
+def test_tensor_core_kernels_with_few_rows_and_padded_rows(n, d, block, kernel):
     """Fewer rows than one group, a ragged last group (also one whose second half is empty), and a leading dimension
     larger than dim: same indices as the general kernel (flips only between neighbours, rarely), same norms, and the
     all-zero row stays on the middle boundary."""
@@ -177,8 +180,8 @@ def test_tensor_core_kernel_with_few_rows_and_padded_rows(n, d, block):
     wide[:, :d] = _dev(xb)
     B.oq_debug_select_rq_kernel(GENERAL)
     ref_idx, ref_norm = B.oq_rotate_quantize_act(wide[:, :d], rot, cb)
-    B.oq_debug_select_rq_kernel(TENSOR)
-    assert B.oq_rq_plan(rot, cb)[0] == TENSOR
+    B.oq_debug_select_rq_kernel(kernel)
+    assert B.oq_rq_plan(rot, cb)[0] == kernel
     idx, norm = B.oq_rotate_quantize_act(wide[:, :d], rot, cb)
     B.oq_debug_select_rq_kernel(AUTO)
     torch.cuda.synchronize()
@@ -243,7 +246,7 @@ def test_empty_and_bad_arguments():
     assert e.value.code == 3
 
 
-@pytest.mark.parametrize("kernel", [AUTO, REGISTERS, TENSOR])
+@pytest.mark.parametrize("kernel", [AUTO, REGISTERS, TENSOR, SLAB])
 def test_results_are_deterministic(kernel):
     import torch
     xb = synth.activations(300, 3072, seed=1001)

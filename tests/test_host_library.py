@@ -123,23 +123,24 @@ def test_level_search_polynomial_counts_boundaries(dim, bits):
             assert dist.max() <= 1e-6 * beta[-1] and np.abs(mag - want)[bad].max() == 1
 
 
-@pytest.mark.parametrize("dim,block,kernel,rows,tiles", [
-    (3072, 128, 3, 16, 3),      # FLUX hidden size: 8 tokens per half group, 192 (token, block) pairs per half
-    (12288, 128, 3, 4, 3),      # FLUX MLP width
-    (5120, 128, 3, 8, 3),       # Wan hidden size: 160 pairs per half
-    (13824, 128, 3, 2, 2),      # Wan FFN width: 108 pairs per half, one tile per half
-    (1024, 128, 2, 16, 0),      # 64 pairs per half would fill half of the tiles: register kernel
-    (3072, 64, 3, 16, 3),       # blocks of 64 and 256 use the same 128-coordinate tile rows
-    (3072, 256, 3, 16, 3),
-    (1024, 256, 2, 8, 0),
-    (3072, 1024, 3, 16, 3),     # the paper's default blocks: same group shapes as blocks of 128
-    (5120, 1024, 3, 8, 3),
-    (12288, 4096, 3, 4, 3),
-    (13824, 512, 3, 2, 2),
-    (1024, 1024, 1, 1, 0),      # a quarter-full tile: general kernel
+@pytest.mark.parametrize("dim,block,kernel,rows,tiles,slab", [
+    (3072, 128, 3, 16, 3, 8),      # FLUX hidden size: 8 tokens per half group, 192 (token, block) pairs per half
+    (12288, 128, 3, 4, 3, 2),      # FLUX MLP width
+    (5120, 128, 3, 8, 3, 4),       # Wan hidden size: 160 pairs per half
+    (13824, 128, 3, 2, 2, 2),      # Wan FFN width: 108 pairs per half, one tile per half
+    (1024, 128, 2, 16, 0, 8),      # 64 pairs per half would fill half of the tiles: register kernel
+    (3072, 64, 3, 16, 3, 8),       # blocks of 64 and 256 use the same 128-coordinate tile rows
+    (3072, 256, 3, 16, 3, 8),
+    (1024, 256, 2, 8, 0, 8),
+    (3072, 1024, 3, 16, 3, 0),     # the paper's default blocks: same group shapes as blocks of 128
+    (5120, 1024, 3, 8, 3, 0),
+    (12288, 4096, 3, 4, 3, 0),
+    (13824, 512, 3, 2, 2, 0),
+    (1024, 1024, 1, 1, 0, 0),      # a quarter-full tile: general kernel
 ])
-def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
-    """Host-side launch planning (no device needed): kernel choice and group shape for the benchmark widths."""
+def test_rotate_quantize_plan(dim, block, kernel, rows, tiles, slab):
+    """Host-side launch planning (no device needed): kernel choice and group shape for the benchmark widths; `slab` =
+    tokens per slab of the token-slab kernel when it is selected (0: it does not take this block size)."""
     rot, cb = B.oq_make_rpbh(dim, block, 0), B.oq_build_codebook(dim, 4)
     k, r, t, smem = B.oq_rq_plan(rot, cb)
     assert (k, r, t) == (kernel, rows, tiles)
@@ -147,6 +148,12 @@ def test_rotate_quantize_plan(dim, block, kernel, rows, tiles):
     B.oq_debug_select_rq_kernel(1)
     try:
         assert B.oq_rq_plan(rot, cb)[0] == 1
+        B.oq_debug_select_rq_kernel(4)
+        k4, r4, t4, smem4 = B.oq_rq_plan(rot, cb)
+        if slab:
+            assert (k4, r4, t4) == (4, slab, 1) and smem4 <= 227 * 1024
+        else:
+            assert k4 != 4                 # falls back
     finally:
         B.oq_debug_select_rq_kernel(0)
 
