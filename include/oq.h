@@ -176,6 +176,41 @@ int oq_linear_forward_noalloc(const void* X_bf16, int n_tokens, int dim, int ldx
                               const oq_codebook* cb_a, const void* Wq_idx, const void* Wq_norm_bf16, int m,
                               const oq_codebook* cb_w, void* Y, int ldy, int y_dtype, void* stream);
 
+/* ---- the linear layers of one transformer block ---------------------------------------------------------- */
+
+/* The method is applied token-wise to every linear layer of a block (Sec. 3.1), and the layers that share an input
+ * dimension share the rotation Pi_d and the activation codebook (Sec. 4.2).  The layers that read the SAME tensor -- the
+ * Q, K and V projections of an attention block -- therefore consume the same quantized activations: one
+ * rotate+quantize pass (Eq. 7-8) feeds all of them.  oq_block_forward runs the layers of a block in the order given, on
+ * one stream, back to back (every kernel is launched with programmatic stream serialisation, so a kernel's set-up
+ * overlaps the tail of the one before it); an input is rotated and quantized once, right before the first layer that reads
+ * it.  Because everything is ordered on the stream, the Y of a layer may be the X of a later input.
+ *   oq_block_input   X_bf16 dev [n_tokens][ldx] bf16; rot / cb_a for its dim; Xq dev scratch owned by the caller:
+ *                    oq_packed_bytes(n_tokens, dim, bits) bytes, or n_tokens * dim * 2 bytes when cb_a has 6 bits (the
+ *                    bf16 level matrix); Xq_norm dev [n_tokens] fp32.  Both hold the quantized input after the call.
+ *   oq_block_layer   input = index into `inputs`; Wq_idx / Wq_norm_bf16 / cb_w from oq_quantize_weights with the input's
+ *                    rotation; Y dev [n_tokens][ldy] of y_dtype.
+ * All arguments are validated before the first launch.  n_tokens == 0 or n_layers == 0 launches nothing.
+ * Errors: as oq_rotate_quantize_act and oq_qlinear (the message names the input or layer). */
+typedef struct {
+  const void* X_bf16;
+  int ldx, dim;
+  const oq_rpbh* rot;
+  const oq_codebook* cb_a;
+  void* Xq;
+  float* Xq_norm;
+} oq_block_input;
+typedef struct {
+  int input, m;
+  const void* Wq_idx;
+  const void* Wq_norm_bf16;
+  const oq_codebook* cb_w;
+  void* Y;
+  int ldy, y_dtype;
+} oq_block_layer;
+int oq_block_forward(int n_tokens, const oq_block_input* inputs, int n_inputs, const oq_block_layer* layers, int n_layers,
+                     void* stream);
+
 /* Test helper: expand packed indices to one byte per coordinate, out dev [rows][dim] uint8, logical level
  * numbers in rotated-coordinate order. */
 int oq_unpack_indices(const void* idx, int rows, int dim, int bits, uint8_t* out, void* stream);

@@ -58,6 +58,7 @@ def lib():
             "oq_adaln_quantize_weights": (i, [vp, i, i, i, vp, vp, vp]),
             "oq_adaln_linear": (i, [vp, i, i, vp, vp, i, i, vp, i, i, vp]),
             "oq_adaln_unpack": (i, [vp, vp, i, i, vp, vp, vp]),
+            "oq_block_forward": (i, [i, vp, i, vp, i, vp]),
             "oq_last_error": (C.c_char_p, []), "oq_version": (C.c_char_p, []),
         }
         for name, (res, args) in sig.items():
@@ -176,6 +177,37 @@ def oq_qlinear(Xq_idx, Xq_norm, cb_a, Wq_idx, Wq_norm, cb_w, dim, out=None, out_
     _check(lib().oq_qlinear(_ptr(Xq_idx), _ptr(Xq_norm), n, cb_a.handle, _ptr(Wq_idx), _ptr(Wq_norm), m,
                             cb_w.handle, dim, _ptr(out), out.stride(0) if n > 1 else m, ydt, _stream()))
     return out
+
+
+class _BlockInput(C.Structure):          # oq_block_input
+    _fields_ = [("X_bf16", C.c_void_p), ("ldx", C.c_int), ("dim", C.c_int), ("rot", C.c_void_p), ("cb_a", C.c_void_p),
+                ("Xq", C.c_void_p), ("Xq_norm", C.c_void_p)]
+
+
+class _BlockLayer(C.Structure):          # oq_block_layer
+    _fields_ = [("input", C.c_int), ("m", C.c_int), ("Wq_idx", C.c_void_p), ("Wq_norm_bf16", C.c_void_p),
+                ("cb_w", C.c_void_p), ("Y", C.c_void_p), ("ldy", C.c_int), ("y_dtype", C.c_int)]
+
+
+def oq_block_forward(inputs, layers):
+    """The linear layers of one block on the current stream; every input is rotated and quantized once.
+    inputs: list of dicts {X (CUDA bf16 [N, d]), rot, cb_a, xq (scratch: packed uint8 [N, pitch], or bf16 [N, d] at 6 bits),
+    xs (fp32 [N])}; layers: list of dicts {input (index), wq, wr, cb_w, Y (CUDA [N, m] bf16 or fp32)}."""
+    import torch
+    n = inputs[0]["X"].shape[0] if inputs else 0
+    ins = (_BlockInput * max(1, len(inputs)))()
+    for k, a in enumerate(inputs):
+        X = a["X"]
+        d = X.shape[1]
+        ins[k] = _BlockInput(X.data_ptr(), X.stride(0) if n > 1 else d, d, a["rot"].handle, a["cb_a"].handle,
+                             a["xq"].data_ptr(), a["xs"].data_ptr())
+    lys = (_BlockLayer * max(1, len(layers)))()
+    for k, l in enumerate(layers):
+        Y = l["Y"]
+        m = Y.shape[1]
+        lys[k] = _BlockLayer(l["input"], m, l["wq"].data_ptr(), l["wr"].data_ptr(), l["cb_w"].handle, Y.data_ptr(),
+                             Y.stride(0) if n > 1 else m, OQ_F32 if Y.dtype == torch.float32 else OQ_BF16)
+    _check(lib().oq_block_forward(n, C.cast(ins, C.c_void_p), len(inputs), C.cast(lys, C.c_void_p), len(layers), _stream()))
 
 
 def oq_forward_workspace_bytes(n_tokens, dim, m, bits_a):

@@ -91,39 +91,30 @@ def run_adaln(n, d, m, iters):
             "gbs": nbytes / med / 1e6, "gbs_best": nbytes / best / 1e6}
 
 
-def run_step(shape, ba, bw, iters):
-    """The four linears of one FLUX- or Wan-shaped block back to back on one stream (rotate+quantize, then GEMM, per
-    layer).  6-bit activations use the bf16-levels operand; 4-bit ones the packed operand."""
+def run_step(shape, ba, bw, iters, split_qkv=False):
+    """The linears of one FLUX- or Wan-shaped block through oq_block_forward (one stream, every input rotated and
+    quantized once).  6-bit activations travel as bf16 levels, 2-4-bit ones packed.  split_qkv: the fused qkv layer
+    becomes three projections that share one quantized input."""
     from . import synth
     tokens, layers = (synth.FLUX_TOKENS, synth.FLUX_LAYERS) if shape == "flux" else (synth.WAN_TOKENS, synth.WAN_LAYERS)
-    L = []
+    inputs, lys = [], []
     for name, d, m in layers:
         rot = B.oq_make_rpbh(d, 128, 0)
         cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
-        W = (torch.randn((m, d), device="cuda") * 0.02).to(torch.bfloat16)
-        wq, wr = B.oq_quantize_weights(W, rot, cbw)
-        del W
-        l = dict(d=d, m=m, rot=rot, cba=cba, cbw=cbw, X=gen_x(tokens, d), wq=wq, wr=wr,
-                 xs=torch.empty(tokens, dtype=torch.float32, device="cuda"),
-                 Y=torch.empty((tokens, m), dtype=torch.bfloat16, device="cuda"))
-        if ba == 6:
-            l["lev"] = torch.empty((tokens, d), dtype=torch.bfloat16, device="cuda")
-        else:
-            l["xq"] = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device="cuda")
-        L.append(l)
-
-    def step():
-        for l in L:
-            if ba == 6:
-                B.oq_rotate_quantize_act_levels(l["X"], l["rot"], l["cba"], out=l["lev"], out_norm=l["xs"])
-                B.oq_qlinear_levels(l["lev"], l["xs"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
-            else:
-                B.oq_rotate_quantize_act(l["X"], l["rot"], l["cba"], out_idx=l["xq"], out_norm=l["xs"])
-                B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
-    med, best = time_kernel(step, iters)
-    fl = sum(2.0 * tokens * l["m"] * l["d"] for l in L)
-    return {"kernel": "block_step", "shape": shape, "tokens": tokens, "bits_a": ba, "bits_w": bw, "ms_median": med,
-            "ms_min": best, "flops": fl, "tflops": fl / med / 1e9, "tflops_best": fl / best / 1e9}
+        xq = (torch.empty((tokens, d), dtype=torch.bfloat16, device="cuda") if ba == 6
+              else torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device="cuda"))
+        inputs.append(dict(X=gen_x(tokens, d), rot=rot, cb_a=cba, xq=xq, xs=torch.empty(tokens, dtype=torch.float32, device="cuda")))
+        for mm in ([m // 3] * 3 if (split_qkv and name == "qkv") else [m]):
+            W = (torch.randn((mm, d), device="cuda") * 0.02).to(torch.bfloat16)
+            wq, wr = B.oq_quantize_weights(W, rot, cbw)
+            del W
+            lys.append(dict(input=len(inputs) - 1, wq=wq, wr=wr, cb_w=cbw, d=d, m=mm,
+                            Y=torch.empty((tokens, mm), dtype=torch.bfloat16, device="cuda")))
+    med, best = time_kernel(lambda: B.oq_block_forward(inputs, lys), iters)
+    fl = sum(2.0 * tokens * l["m"] * l["d"] for l in lys)
+    return {"kernel": "block_step", "shape": shape, "tokens": tokens, "bits_a": ba, "bits_w": bw, "layers": len(lys),
+            "inputs": len(inputs), "ms_median": med, "ms_min": best, "flops": fl, "tflops": fl / med / 1e9,
+            "tflops_best": fl / best / 1e9}
 
 
 def main(argv=None):
@@ -140,6 +131,7 @@ def main(argv=None):
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--shape", choices=["flux", "wan"], default="wan")
     ap.add_argument("--levels", action="store_true", help="gemm: activations as bf16 levels (oq_qlinear_levels)")
+    ap.add_argument("--split-qkv", action="store_true", help="step: q, k, v as three layers that share one quantized input")
     ap.add_argument("--kernel", type=int, default=0, help="rotate+quantize kernel: 0 auto, 1 general, 2 registers, 3 tensor cores")
     a = ap.parse_args(argv)
     oqbuild.build()
@@ -149,7 +141,7 @@ def main(argv=None):
     elif a.mode == "gemm":
         print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters, a.levels)))
     elif a.mode == "step":
-        print(json.dumps(run_step(a.shape, a.bits_a, a.bits_w, a.iters)))
+        print(json.dumps(run_step(a.shape, a.bits_a, a.bits_w, a.iters, a.split_qkv)))
     elif a.mode == "adaln":
         print(json.dumps(run_adaln(a.tokens, a.dim, a.m, a.iters)))
     else:
