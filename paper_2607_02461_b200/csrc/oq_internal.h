@@ -87,7 +87,7 @@ inline uint32_t rq_mm_chunk_offset(int i, int tok, int nb) {
   return 16u * (uint32_t)row + (uint32_t)(h * 2 * tok);
 }
 struct RqMmShape {
-  int tok, seg_rows, pad_rows, nstages, tab_smem, mask_smem;
+  int tok, seg_rows, pad_rows, tab_smem, mask_smem;
   size_t smem;
 };
 // false: this width does not run on the token-slab kernel.  The largest slab that fits in shared memory beside the
@@ -100,6 +100,7 @@ inline bool rq_mm_shape(int dim, RqMmShape* shape) {
   for (int tok = 8; tok >= 2; tok >>= 1) {
     const int hw = 8 / tok, bc = 128 / tok;
     if (dim % (32 * hw)) continue;
+    if (dim / (32 * hw) > 128) continue;       // 16 front-end warps x 8 windows in registers per slab
     if (!(nb >= bc - 1 || (bc % nb == 0 && bc / nb <= 2))) continue;
     const int raw = nb * tok, seg_rows = (raw + 15) / 16 * 16;
     if (seg_rows > 16383) continue;
@@ -111,7 +112,7 @@ inline bool rq_mm_shape(int dim, RqMmShape* shape) {
       const size_t smem = 1024 + 65536 + 2 * slab + (tab ? 4 * (size_t)dim : 0) + (mask ? 2 * (size_t)dim : 0) + 3072;
       if (smem <= kMaxSmem) {
         shape->tok = tok; shape->seg_rows = seg_rows; shape->pad_rows = seg_rows - raw;
-        shape->nstages = 0; shape->tab_smem = tab; shape->mask_smem = mask; shape->smem = smem;
+        shape->tab_smem = tab; shape->mask_smem = mask; shape->smem = smem;
         return true;
       }
     }

@@ -189,7 +189,6 @@ static cudaError_t launch_fast_T(int bits, int grid, const FastPlan& pl, cudaStr
 // row-per-thread one on every benchmark shape), 1 = general, 2 = register butterflies, 3 = tensor cores (row-per-thread
 // gather), 4 = tensor cores (token-slab gather).  A forced kernel that cannot handle the shape falls back.
 static int g_forced_kernel = 0;
-static int g_mm_desc_swap = 0;      // test switch of the token-slab kernel's operand descriptors
 
 // Token-slab kernel: blocks of 64, 128, 256; packed outputs; widths for which rq_mm_shape finds a slab size.
 static bool plan_mm(int dim, int block, const oq_codebook* cb, RqMmShape* shape) {
@@ -285,9 +284,8 @@ static int launch_rq(const char* fn, const void* X, int rows, int dim, int ld, c
     prm.out_norm = out_norm; prm.dbg = dbg; prm.poly = cb->poly;
     prm.nslabs = (rows + ms.tok - 1) / ms.tok;
     prm.nb = dim / 128;
-    prm.seg_rows = ms.seg_rows; prm.pad_rows = ms.pad_rows; prm.nstages = ms.nstages; prm.tab_smem = ms.tab_smem; prm.mask_smem = ms.mask_smem;
+    prm.seg_rows = ms.seg_rows; prm.pad_rows = ms.pad_rows; prm.tab_smem = ms.tab_smem; prm.mask_smem = ms.mask_smem;
     prm.bf16_norm = kBf16Norm ? 1 : 0;
-    prm.desc_swap = g_mm_desc_swap;
     prm.status = status;
     const int grid = sms < prm.nslabs ? sms : prm.nslabs;
     e = rq_mm_launch(cb->bits, ms.tok, rot->block, grid, ms.smem, st, prm);
@@ -461,10 +459,6 @@ int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows
 }
 
 int oq_debug_select_rq_kernel(int which) {
-  if (which >= 100 && which <= 101) {      // 100 / 101: stride fields of the token-slab kernel's descriptors as built / exchanged
-    g_mm_desc_swap = which - 100;
-    return OQ_OK;
-  }
   if (which < 0 || which > 4) return fail(OQ_ERR_INVALID_ARG, "oq_debug_select_rq_kernel: which must be 0..4");
   g_forced_kernel = which;
   return OQ_OK;

@@ -14,15 +14,14 @@
 // therefore known before the first of its tiles is quantized, and every accumulator is read exactly once.
 //
 // Pipeline of one CTA (one per SM, persistent over its slabs; every wait is bounded and reports to a status word):
-//   loader (8 w)  global rows -> 16 bytes per lane (12 loads in flight per thread, issued before the slab buffer is
-//                 free) -> sign flips by SOURCE position -> stmatrix.trans -> slab buffer
+//   front end (16 w)  per slab: the rows of the NEXT slab are already in registers (16-byte global loads issued a slab
+//                 ahead); sign flips by SOURCE position -> stmatrix.trans -> slab buffer; named barrier; then the tiles
+//                 that the slab completes: table look-up of the chunk address, one load + one store per chunk into
+//                 the operand tile (two halves of 64 coordinates, refilled as soon as their MMAs have completed)
 //   MMA (1 thr)   Gram product of a slab; per tile 8 x tcgen05.mma (M = 128 pairs, N = 128, K = 16) into one of
 //                 three accumulators
-//   gather (4 w)  per tile: table look-up of the chunk address, one load + one store per chunk into the operand
-//                 tile (two halves of 64 coordinates, refilled as soon as their MMAs have completed); per slab: the
-//                 diagonal of the Gram matrix -> norms
-//   compute (16 w, two groups of 8 that take alternate tiles) reads 2 x 32 accumulator columns per thread, finds the
-//                 level with the polynomial of QuantPoly, packs and stores.
+//   compute (8 w) per slab: the diagonal of the Gram matrix -> norms; per tile: 2 x 32 accumulator columns per thread,
+//                 level search with the polynomial of QuantPoly, packing, stores.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -34,43 +33,28 @@
 namespace oq {
 
 namespace rqmm {
-#ifndef OQ_RQMM_COMPUTE_WARPS
-#define OQ_RQMM_COMPUTE_WARPS 8
-#endif
-#ifndef OQ_RQMM_LOADER_WARPS
-#define OQ_RQMM_LOADER_WARPS 8
-#endif
-#ifndef OQ_RQMM_PIECES
-#define OQ_RQMM_PIECES 2
-#endif
-constexpr int COMPUTE_WARPS = OQ_RQMM_COMPUTE_WARPS, GATHER_WARPS = 4, LOADER_WARPS = OQ_RQMM_LOADER_WARPS;
-constexpr int LOAD_BATCH = 12;                    // 16-byte global loads one loader thread keeps in flight
-constexpr int PIECES = OQ_RQMM_PIECES;            // pieces of 32 accumulator columns one compute thread handles per tile
-constexpr int WARPS_PER_TILE = 4 * (4 / PIECES);  // 4 lane quarters x column parts
-constexpr int GROUPS = COMPUTE_WARPS / WARPS_PER_TILE;   // group g of compute warps takes the tiles i = g mod GROUPS
-static_assert(COMPUTE_WARPS % WARPS_PER_TILE == 0 && GATHER_WARPS == 4 && COMPUTE_WARPS % 4 == 0,
-              "warp roles: gather warp g must sit in lane quarter g of tensor memory");
-constexpr int GATHER_WARP0 = COMPUTE_WARPS, LOADER_WARP0 = GATHER_WARP0 + GATHER_WARPS, MMA_WARP = LOADER_WARP0 + LOADER_WARPS;
+constexpr int COMPUTE_WARPS = 8, FE_WARPS = 16;
+constexpr int PIECES = 2;                         // pieces of 32 accumulator columns one compute thread handles per tile
+constexpr int FE_WARP0 = COMPUTE_WARPS, MMA_WARP = FE_WARP0 + FE_WARPS;
 constexpr int THREADS = (MMA_WARP + 1) * 32;
 constexpr int SLOTS = 3;                          // accumulators of 128 columns
 constexpr uint32_t GRAM_COL = SLOTS * 128;        // Gram accumulator
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t ATOM = 128 * 128;              // one 64-coordinate half of the K-major, 128-byte-swizzled H tile
 constexpr uint32_t OFF_H = 0, OFF_A = 32768, OFF_T = 65536;   // H tile, operand tile, two slab buffers
-constexpr int NORM_RING = 16;
-enum { B_TFULL = 0, B_TFREE = 2, B_AFULL = 4, B_AFREE = 6, B_ACCRDY = 8, B_ACCFREE = 11, B_GRAMRDY = 14,
-       B_GRAMFREE = 15, B_NORM = 16, NBARS = 16 + NORM_RING };
-enum { WAIT_STAGE = 21, WAIT_TFULL = 22, WAIT_TFREE = 23, WAIT_AFULL = 24, WAIT_AFREE = 25, WAIT_ACC = 26,
-       WAIT_ACCFREE = 27, WAIT_GRAM = 28, WAIT_GRAMFREE = 29, WAIT_NORM = 30, WAIT_DRAIN = 31, WAIT_STGFREE = 32 };
+constexpr int WIN_SLOTS = 8;                      // 16-byte global loads one front-end thread keeps in flight
+constexpr int NORM_RING = 4;
+enum { B_TFULL = 0, B_TDONE = 2, B_AFULL = 4, B_AFREE = 6, B_ACCRDY = 8, B_ACCFREE = 11, B_GRAMRDY = 14, B_GRAMFREE = 15, NBARS = 16 };
+enum { WAIT_TFULL = 22, WAIT_TDONE = 23, WAIT_AFULL = 24, WAIT_AFREE = 25, WAIT_ACC = 26, WAIT_ACCFREE = 27, WAIT_GRAM = 28,
+       WAIT_GRAMFREE = 29 };
 __host__ __device__ constexpr int window_row(int cb) { return rq_mm_window_row(cb); }
 }  // namespace rqmm
 
 // Shared-memory matrix descriptor of an MN-major operand with the 128-byte swizzle: atoms of 64 elements along M/N
 // (128 contiguous bytes, 16-byte pieces XOR-ed with the row number) x 8 rows along K; `mn_stride` bytes between atoms
 // that are neighbours along M/N, `k_stride` bytes between neighbours along K.
-__device__ __forceinline__ uint64_t mn_major_desc(uint32_t addr, uint32_t mn_stride, uint32_t k_stride, int swap) {
-  const uint32_t lbo = swap ? k_stride : mn_stride, sbo = swap ? mn_stride : k_stride;
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) | ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) |
+__device__ __forceinline__ uint64_t mn_major_desc(uint32_t addr, uint32_t mn_stride, uint32_t k_stride) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((mn_stride >> 4) & 0x3FFFu) << 16) | ((uint64_t)((k_stride >> 4) & 0x3FFFu) << 32) |
          (1ull << 46) | (2ull << 61);
 }
 
@@ -80,8 +64,8 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
   constexpr int CB = 2 * TOK;            // chunk bytes
   constexpr int SUBS = 8 / TOK;          // chunks per 16-byte row
   constexpr int BC = 128 / TOK;          // (slab, block) chunks of 128 rotated coordinates per tile
-    constexpr int GPW = TOK / 2;           // groups of 8 * SUBS lanes per gather warp
-  constexpr int PASSES = 4 / GPW;        // passes of the gather warps over the 16 core-matrix columns of a tile
+  constexpr int GPW = TOK / 2;           // groups of 8 * SUBS lanes per front-end warp
+  constexpr int PASSES = 4 / GPW;        // passes over the 16 piece columns of the operand tile
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
@@ -90,9 +74,8 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
   const uint32_t tab_base = t_base + 2 * slab_bytes;
   const uint32_t msk_base = tab_base + (p.tab_smem ? 4u * (uint32_t)p.dim : 0u);
   unsigned char* small = smem + (msk_base - sbase) + (p.mask_smem ? 2u * (uint32_t)p.dim : 0u);
-  float* s_diag = reinterpret_cast<float*>(small);                       // [2][128]
-  float* s_norm = s_diag + 256;                                          // [NORM_RING][8]: norms of the last slabs
-  uint64_t* bars = reinterpret_cast<uint64_t*>(s_norm + NORM_RING * 8);
+  float* s_part = reinterpret_cast<float*>(small);                       // [NORM_RING][4 lane quarters][8 row elements]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(s_part + NORM_RING * 32);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NBARS + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar0 = smem_u32(bars);
@@ -106,18 +89,17 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(B_TFULL + i), LOADER_WARPS);
-      mbar_init(bar(B_TFREE + i), GATHER_WARPS + 1);
-      mbar_init(bar(B_AFULL + i), GATHER_WARPS);
+      mbar_init(bar(B_TFULL + i), 1);
+      mbar_init(bar(B_TDONE + i), 1);
+      mbar_init(bar(B_AFULL + i), FE_WARPS / 2);
       mbar_init(bar(B_AFREE + i), 1);
     }
     for (int i = 0; i < SLOTS; ++i) {
       mbar_init(bar(B_ACCRDY + i), 1);
-      mbar_init(bar(B_ACCFREE + i), COMPUTE_WARPS / GROUPS);
+      mbar_init(bar(B_ACCFREE + i), COMPUTE_WARPS);
     }
     mbar_init(bar(B_GRAMRDY), 1);
-    mbar_init(bar(B_GRAMFREE), GATHER_WARPS);
-    for (int i = 0; i < NORM_RING; ++i) mbar_init(bar(B_NORM + i), 1);
+    mbar_init(bar(B_GRAMFREE), 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -176,43 +158,13 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
   const uint32_t tmem = *tmem_slot;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-#ifdef OQ_RQMM_TIMING
-  // instrumented build: lane 0 of every warp adds up the cycles it spends in each kind of wait; p.dbg receives
-  // [CTA][warp][16] 64-bit counters (slot 15: the warp's whole loop) instead of rotated values
-  // (few counters: 0 = all waits, 1..3 = sections of the role, so that the instrumentation costs few registers)
-  long long tw[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) tw[i] = 0;
-  const long long t_begin = clock64();
-#define OQ_TW_BEGIN const long long tw0 = clock64();
-#define OQ_TW_END(code) tw[0] += clock64() - tw0;
-#define OQ_SEC_BEGIN(name) const long long name = clock64();
-#define OQ_SEC_END(name, slot) if (lane == 0) tw[(slot) - 9] += clock64() - name;
-#else
-#define OQ_TW_BEGIN
-#define OQ_TW_END(code)
-#define OQ_SEC_BEGIN(name)
-#define OQ_SEC_END(name, slot)
-#endif
 #ifdef OQ_RQMM_TRACE
   // trace build: CTA 0 records clock64 at pipeline events, p.dbg receives [16 kinds][64 events] 64-bit stamps
 #define OQ_EV(kind, idx) if (blockIdx.x == 0 && lane == 0 && (idx) < 64 && p.dbg != nullptr) reinterpret_cast<long long*>(p.dbg)[(kind) * 64 + (idx)] = clock64();
-// the same, but the clock is read only after `dep` (a 32-bit value) is available
-#define OQ_EV_AFTER(kind, idx, dep) { long long tdep; asm volatile("mov.u64 %0, %%clock64;" : "=l"(tdep) : "r"(dep)); \
-  if (blockIdx.x == 0 && lane == 0 && (idx) < 64 && p.dbg != nullptr) reinterpret_cast<long long*>(p.dbg)[(kind) * 64 + (idx)] = tdep; }
 #else
 #define OQ_EV(kind, idx)
-#define OQ_EV_AFTER(kind, idx, dep)
 #endif
-  auto wait1 = [&](uint32_t b, uint32_t parity, int code) {
-    OQ_TW_BEGIN
-#ifdef OQ_RQMM_SLEEP_NS
-    mbar_wait(b, parity, abort_flag, p.status, code, WAIT_CYCLES, OQ_RQMM_SLEEP_NS);
-#else
-    mbar_wait(b, parity, abort_flag, p.status, code);
-#endif
-    OQ_TW_END(code)
-  };
+  auto wait1 = [&](uint32_t b, uint32_t parity, int code) { mbar_wait(b, parity, abort_flag, p.status, code); };
   auto warp_wait = [&](uint32_t b, uint32_t parity, int code) {
     if (lane == 0) wait1(b, parity, code);
     __syncwarp();
@@ -251,7 +203,7 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
           OQ_EV(3, s)
           const uint32_t tb = t_base + (uint32_t)(s & 1) * slab_bytes;
           for (int g = 0; g < ngram; ++g) {
-            const uint64_t dsc = mn_major_desc(tb + 2048u * (uint32_t)g, 128u * (uint32_t)p.seg_rows, 1024u, p.desc_swap);
+            const uint64_t dsc = mn_major_desc(tb + 2048u * (uint32_t)g, 128u * (uint32_t)p.seg_rows, 1024u);
             const uint32_t acc = g > 0 ? 1u : 0u;
             asm volatile(
                 "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
@@ -259,7 +211,7 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
                 ::"r"(tmem + GRAM_COL), "l"(dsc), "l"(dsc), "r"(IDESC_G), "r"(acc) : "memory");
           }
           asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar(B_GRAMRDY)) : "memory");
-          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar(B_TFREE + (s & 1))) : "memory");
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar(B_TDONE + (s & 1))) : "memory");
         }
         const uint32_t slot = (uint32_t)i % 3u, use = (uint32_t)i / 3u;
         if (use > 0u) wait1(bar(B_ACCFREE + slot), (use - 1u) & 1u, WAIT_ACCFREE);
@@ -270,7 +222,7 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
           for (int k4 = 4 * half; k4 < 4 * half + 4; ++k4) {
-            const uint64_t da = mn_major_desc(a_base + 4096u * (uint32_t)k4, 1024u, 2048u, p.desc_swap);
+            const uint64_t da = mn_major_desc(a_base + 4096u * (uint32_t)k4, 1024u, 2048u);
             const uint64_t db = desc_h + (uint64_t)((k4 >> 2) * (ATOM >> 4)) + 2 * (k4 & 3);
             const uint32_t acc = k4 > 0 ? 1u : 0u;
             asm volatile(
@@ -284,210 +236,210 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
         OQ_EV(5, i)
       }
     }
-  } else if (warp >= LOADER_WARP0) {
-    // ------------------------------- loader warps: global rows -> transposed slab -------------------------------
-    const int lw = warp - LOADER_WARP0;
-    const int frow = lane >> 2;                               // row of the 8 x 8 fragments this lane holds
+  } else if (warp >= FE_WARP0) {
+    // ------------------------------- front end: global rows -> transposed slab -> operand tiles -------------------------------
+    const int fw = warp - FE_WARP0;
+    // as loader: lane = (fragment row, 8 coordinates); as provider of a row address: matrix lane / 8, transposed row lane % 8
+    const int frow = lane >> 2;
     const int tok = frow % TOK, h = frow / TOK;               // its token, its 32-coordinate sub-window
-    const int c8 = (lane & 3) * 8;                            // its 8 coordinates inside the sub-window
-    // as provider of a row address: matrix m = lane / 8, transposed row c' = lane % 8
+    const int c8 = (lane & 3) * 8;
     const int cb_addr = ((lane & 7) >> 1) * 8 + 2 * (lane >> 3) + (lane & 1);
     const int wrow = window_row(cb_addr);
     const int nwin = p.dim / (32 * SUBS);                     // windows of 32 * SUBS coordinates per row
-    const int coord_thr = lw * 32 * SUBS + h * 32 + c8;       // this lane's coordinates in the warp's first window
+    const int coord_thr = fw * 32 * SUBS + h * 32 + c8;       // this lane's coordinates in the warp's first window
+    // as gatherer: piece column mm of the tile (per pass), coordinates k = 8 kg + kr with kg in [4 kq, 4 kq + 4)
+    const int gw = fw & 3, kq = fw >> 2, half = kq >> 1;
+    const int sub = lane % SUBS, kr = (lane / SUBS) & 7, grp = lane / (8 * SUBS);
+    const uint32_t tab_thr = (uint32_t)kr * 16u + 4u * (uint32_t)kq;     // + j * 128: 4 consecutive entries
+    uint32_t r[WIN_SLOTS][4];
+    auto load_slab = [&](int sl) {        // the warp's windows fw, fw + FE_WARPS, ... of slab sl -> registers
+      const int row = ((int)blockIdx.x + sl * stride) * TOK + tok;
+      const bool row_ok = sl < nsl && row < p.rows;
+      const unsigned char* src = p.X + ((size_t)(row_ok ? row : 0) * p.ldx + coord_thr) * 2;
+#pragma unroll
+      for (int u = 0; u < WIN_SLOTS; ++u) {
+        r[u][0] = r[u][1] = r[u][2] = r[u][3] = 0u;
+        if (row_ok && fw + u * FE_WARPS < nwin)
+          asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[u][0]), "=r"(r[u][1]), "=r"(r[u][2]), "=r"(r[u][3])
+                       : "l"(src + (size_t)u * (FE_WARPS * 64 * SUBS)));
+      }
+    };
+    // Rows reach the registers through L2: one thread asks for the rows of a slab two slabs before they are loaded, so
+    // that the loads (issued right after a slab has been stored, used one slab later) are short when the next fence of
+    // this thread has to wait for them.
+    auto prefetch_slab = [&](int sl) {
+      if (sl >= nsl) return;
+      const int row0 = ((int)blockIdx.x + sl * stride) * TOK;
+      for (int rr = 0; rr < TOK && row0 + rr < p.rows; ++rr)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.X + (size_t)(row0 + rr) * p.ldx * 2), "r"(2u * (uint32_t)p.dim) : "memory");
+    };
+    if (fw == 1 && lane == 0) {
+      prefetch_slab(1);
+      prefetch_slab(2);
+    }
+    load_slab(0);
+    int next_tile = 0;
+    int sl0 = 0, j0 = 0;                             // first chunk of tile next_tile
     for (int sl = 0; sl < nsl; ++sl) {
       const uint32_t tb = t_base + (uint32_t)(sl & 1) * slab_bytes;
-      const int row = ((int)blockIdx.x + sl * stride) * TOK + tok;
-      const bool row_ok = row < p.rows;
-      const unsigned char* src = p.X + ((size_t)(row_ok ? row : 0) * p.ldx + coord_thr) * 2;
-      // The warp takes the windows lw, lw + LOADER_WARPS, ... of the slab, LOAD_BATCH at a time: all global loads of a
-      // batch first (the first batch is issued before the slab buffer is known to be free: the data waits in
-      // registers), then the sign flips and the transposing stores.
-      for (int u0 = 0; lw + u0 * LOADER_WARPS < nwin; u0 += LOAD_BATCH) {
-        uint32_t r[LOAD_BATCH][4];
+      // the buffer held slab sl - 2: its Gram product must have been read by the tensor cores, and every front-end warp
+      // must have finished the tiles that gathered from it (they were gathered before this point of the program)
+      if (sl >= 2) warp_wait(bar(B_TDONE + (sl & 1)), (uint32_t)((sl >> 1) - 1) & 1u, WAIT_TDONE);
+      if (sl >= 1) asm volatile("bar.sync 2, %0;" ::"n"(FE_WARPS * 32) : "memory");
+      if (fw == 0) { OQ_EV(0, sl) }
+      // sign flips first (the mask loads of all windows are in flight together), then the transposing stores
 #pragma unroll
-        for (int u = 0; u < LOAD_BATCH; ++u) {
-          r[u][0] = r[u][1] = r[u][2] = r[u][3] = 0u;
-          if (row_ok && lw + (u0 + u) * LOADER_WARPS < nwin)
-            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r[u][0]), "=r"(r[u][1]), "=r"(r[u][2]), "=r"(r[u][3])
-                         : "l"(src + (size_t)(u0 + u) * (LOADER_WARPS * 64 * SUBS)));
+      for (int u = 0; u < WIN_SLOTS; ++u) {
+        if (fw + u * FE_WARPS < nwin) {
+          const int coord = coord_thr + u * (FE_WARPS * 32 * SUBS);
+          uint4 m;
+          if (p.mask_smem)
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w) : "r"(msk_base + 2u * (uint32_t)coord));
+          else
+            m = __ldg(reinterpret_cast<const uint4*>(p.srcmask + (coord >> 1)));
+          r[u][0] ^= m.x; r[u][1] ^= m.y; r[u][2] ^= m.z; r[u][3] ^= m.w;
         }
-        if (u0 == 0 && sl >= 2) warp_wait(bar(B_TFREE + (sl & 1)), (uint32_t)((sl >> 1) - 1) & 1u, WAIT_TFREE);
-        if (lw == 0) { OQ_EV(0, sl) }
-#pragma unroll
-        for (int u = 0; u < LOAD_BATCH; ++u) {
-          if (lw + (u0 + u) * LOADER_WARPS < nwin) {
-            const int coord = coord_thr + (u0 + u) * (LOADER_WARPS * 32 * SUBS);
-            uint4 m;
-            if (p.mask_smem)
-              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w) : "r"(msk_base + 2u * (uint32_t)coord));
-            else
-              m = __ldg(reinterpret_cast<const uint4*>(p.srcmask + (coord >> 1)));
-            int lin = (lw + (u0 + u) * LOADER_WARPS) * 32 + wrow;      // row of the slab buffer before padding
-            if (lin >= 8 * raw_rows) lin += 8 * p.pad_rows;
-            asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};"
-                         ::"r"(tb + 16u * (uint32_t)lin), "r"(r[u][0] ^ m.x), "r"(r[u][1] ^ m.y), "r"(r[u][2] ^ m.z), "r"(r[u][3] ^ m.w) : "memory");
-          }
-        }
-        if (lw == 0) { OQ_EV(1, sl) }
       }
-      if (lw == 0) { OQ_EV(2, sl) }
+#pragma unroll
+      for (int u = 0; u < WIN_SLOTS; ++u) {
+        if (fw + u * FE_WARPS < nwin) {
+          int lin = (fw + u * FE_WARPS) * 32 + wrow;          // row of the slab buffer before padding
+          if (lin >= 8 * raw_rows) lin += 8 * p.pad_rows;
+          asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};"
+                       ::"r"(tb + 16u * (uint32_t)lin), "r"(r[u][0]), "r"(r[u][1]), "r"(r[u][2]), "r"(r[u][3]) : "memory");
+        }
+      }
       // the tensor cores read the slab buffer (Gram product): make this thread's writes visible to the async proxy
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_TFULL + (sl & 1))) : "memory");
-    }
-  } else if (warp >= GATHER_WARP0) {
-    // ------------------------------- gather warps -------------------------------
-    const int gw = warp - GATHER_WARP0;
-    const int sub = lane % SUBS, kr = (lane / SUBS) & 7, grp = lane / (8 * SUBS);
-    const uint32_t tab_thr = (uint32_t)kr * 16u;               // + j * 128 + half * 8: 8 consecutive entries
-    int next_norm = 0;
-    int sl0 = 0, j0 = 0;                             // first chunk of tile i
-    for (int i = 0; i < ntiles; ++i) {
-      const int sl_last = tile_last_slab(sl0, j0);
-      warp_wait(bar(B_TFULL + (sl_last & 1)), (uint32_t)(sl_last >> 1) & 1u, WAIT_TFULL);
-      if (gw == 0) { OQ_EV(8, i) }
-      // the chunks this thread moves: one per pass (core-matrix column mm of the tile), 16 coordinates k = 8 kg + kr each
-      int mmv[PASSES];
-      uint32_t srcb[PASSES], tabj[PASSES];
-      bool okv[PASSES];
-#pragma unroll
-      for (int ps = 0; ps < PASSES; ++ps) {
-        const int mm = ps * (GATHER_WARPS * GPW) + gw * GPW + grp;
-        int sl = sl0, j = j0;
-        advance(sl, j, mm * SUBS + sub);
-        mmv[ps] = mm;
-        okv[ps] = sl < nsl;
-        srcb[ps] = t_base + (uint32_t)(sl & 1) * slab_bytes;
-        tabj[ps] = (uint32_t)j * 128u + tab_thr;
+      asm volatile("bar.sync 3, %0;" ::"n"(FE_WARPS * 32) : "memory");
+      if (fw == 0) {
+        OQ_EV(2, sl)
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_TFULL + (sl & 1))) : "memory");
       }
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      if (fw == 1 && lane == 0) prefetch_slab(sl + 3);
+      load_slab(sl + 1);                               // from L2; used when the next slab is stored
+      // the tiles that this slab completes
+      while (next_tile < ntiles && tile_last_slab(sl0, j0) == sl) {
+        const int i = next_tile;
+        if (fw == 0) { OQ_EV(8, i) }
         if (i > 0) warp_wait(bar(B_AFREE + half), (uint32_t)(i - 1) & 1u, WAIT_AFREE);
-        OQ_SEC_BEGIN(sec_gm)
 #pragma unroll
         for (int ps = 0; ps < PASSES; ++ps) {
-          if (okv[ps]) {
-            uint32_t off[8];
+          const int mm = ps * (4 * GPW) + gw * GPW + grp;
+          int s2 = sl0, j = j0;
+          advance(s2, j, mm * SUBS + sub);
+          if (s2 < nsl) {
+            uint32_t off[4];
             if (p.tab_smem) {
-              const uint32_t ta = tab_base + 4u * (tabj[ps] + 8u * half);
-              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(off[0]), "=r"(off[1]), "=r"(off[2]), "=r"(off[3]) : "r"(ta));
-              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(off[4]), "=r"(off[5]), "=r"(off[6]), "=r"(off[7]) : "r"(ta + 16u));
+              asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(off[0]), "=r"(off[1]), "=r"(off[2]), "=r"(off[3])
+                           : "r"(tab_base + 4u * ((uint32_t)j * 128u + tab_thr)));
             } else {
-              const uint4* tg = reinterpret_cast<const uint4*>(p.table + tabj[ps] + 8 * half);
-              const uint4 o0 = __ldg(tg), o1 = __ldg(tg + 1);
-              off[0] = o0.x; off[1] = o0.y; off[2] = o0.z; off[3] = o0.w;
-              off[4] = o1.x; off[5] = o1.y; off[6] = o1.z; off[7] = o1.w;
+              const uint4 o = __ldg(reinterpret_cast<const uint4*>(p.table + (uint32_t)j * 128u + tab_thr));
+              off[0] = o.x; off[1] = o.y; off[2] = o.z; off[3] = o.w;
             }
-            // operand tile: [8 coordinates k / 8][2 halves of the 128 rows][k % 8][8 pieces of 16 bytes, XOR-ed with k % 8]
-            const uint32_t dst = a_base + (uint32_t)half * 16384u + (uint32_t)(mmv[ps] >> 3) * 1024u + (uint32_t)kr * 128u +
-                                 (uint32_t)(((mmv[ps] & 7) ^ kr) << 4) + (uint32_t)sub * CB;
+            const uint32_t srcb = t_base + (uint32_t)(s2 & 1) * slab_bytes;
+            // operand tile: [coordinates k / 8][2 halves of the 128 rows][k % 8][8 pieces of 16 bytes, XOR-ed with k % 8]
+            const uint32_t dst = a_base + (uint32_t)(4 * kq) * 2048u + (uint32_t)(mm >> 3) * 1024u + (uint32_t)kr * 128u +
+                                 (uint32_t)(((mm & 7) ^ kr) << 4) + (uint32_t)sub * CB;
             if constexpr (TOK == 8) {
-              uint4 c[8];
+              uint4 c[4];
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk)
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(c[kk].x), "=r"(c[kk].y), "=r"(c[kk].z), "=r"(c[kk].w) : "r"(srcb[ps] + off[kk]));
+              for (int kk = 0; kk < 4; ++kk)
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(c[kk].x), "=r"(c[kk].y), "=r"(c[kk].z), "=r"(c[kk].w) : "r"(srcb + off[kk]));
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk)
+              for (int kk = 0; kk < 4; ++kk)
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst + 2048u * kk), "r"(c[kk].x), "r"(c[kk].y), "r"(c[kk].z), "r"(c[kk].w) : "memory");
             } else if constexpr (TOK == 4) {
-              uint2 c[8];
+              uint2 c[4];
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk)
-                asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(c[kk].x), "=r"(c[kk].y) : "r"(srcb[ps] + off[kk]));
+              for (int kk = 0; kk < 4; ++kk) asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(c[kk].x), "=r"(c[kk].y) : "r"(srcb + off[kk]));
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk)
-                asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(dst + 2048u * kk), "r"(c[kk].x), "r"(c[kk].y) : "memory");
+              for (int kk = 0; kk < 4; ++kk) asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(dst + 2048u * kk), "r"(c[kk].x), "r"(c[kk].y) : "memory");
             } else {
-              uint32_t c[8];
+              uint32_t c[4];
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(c[kk]) : "r"(srcb[ps] + off[kk]));
+              for (int kk = 0; kk < 4; ++kk) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(c[kk]) : "r"(srcb + off[kk]));
 #pragma unroll
-              for (int kk = 0; kk < 8; ++kk) asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst + 2048u * kk), "r"(c[kk]) : "memory");
+              for (int kk = 0; kk < 4; ++kk) asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst + 2048u * kk), "r"(c[kk]) : "memory");
             }
           }
         }
-        OQ_SEC_END(sec_gm, 11)
-        OQ_SEC_BEGIN(sec_gf)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        OQ_SEC_END(sec_gf, 12)
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_AFULL + half)) : "memory");
-      }
-      if (gw == 0) { OQ_EV(9, i) }
-      // slabs whose last chunk lies in this tile are no longer needed by this warp
-      const int first = sl0;
-      advance(sl0, j0, BC);                          // now the first chunk of the next tile
-      if (lane == 0) {
-        for (int sl = first; sl < sl0 && sl < nsl; ++sl)
-          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_TFREE + (sl & 1))) : "memory");
-      }
-      // norms of the slabs that this tile is the first to touch: diagonal of the Gram matrix (whose product ran on the
-      // tensor cores while the tile was gathered)
-      for (; next_norm <= sl_last; ++next_norm) {
-        const int s = next_norm;
-        warp_wait(bar(B_GRAMRDY), (uint32_t)s & 1u, WAIT_GRAM);
-        if (gw == 0) { OQ_EV(6, s) }
-        OQ_SEC_BEGIN(sec_gn)
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t v[32];
-        tmem_load32(tmem + ((uint32_t)(gw * 32) << 16) + GRAM_COL + (uint32_t)gw * 32u, v);
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_GRAMFREE)) : "memory");
-        // entry (lane, lane) of the warp's 32 x 32 diagonal block
-#pragma unroll
-        for (int hb = 16; hb >= 1; hb >>= 1) {
-          const bool up = (lane & hb) != 0;
-#pragma unroll
-          for (int e = 0; e < hb; ++e) v[e] = up ? v[e + hb] : v[e];
-        }
-        float* dg = s_diag + (s & 1) * 128;
-        dg[gw * 32 + lane] = __uint_as_float(v[0]);
-        asm volatile("bar.sync 2, %0;" ::"n"(GATHER_WARPS * 32) : "memory");
-        if (gw == 0) {
-          if (lane < TOK) {
-            // rows of the Gram matrix that belong to token `lane`: element h * TOK + lane of every 16-byte row group
-            float tot = 0.f;
-#pragma unroll
-            for (int c = 0; c < 16; ++c)
-#pragma unroll
-              for (int hh = 0; hh < SUBS; ++hh) tot += dg[c * 8 + hh * TOK + lane];
-            const float nrm = sqrtf(tot);
-            s_norm[(s & (NORM_RING - 1)) * 8 + lane] = nrm;
-            const long long row = ((long long)blockIdx.x + (long long)s * stride) * TOK + lane;
-            if (row < p.rows) {
-              if (p.bf16_norm) reinterpret_cast<__nv_bfloat16*>(p.out_norm)[row] = __float2bfloat16_rn(nrm);
-              else reinterpret_cast<float*>(p.out_norm)[row] = nrm;
-            }
-          }
-          __syncwarp();
-          if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_NORM + (s & (NORM_RING - 1)))) : "memory");
-        }
-        OQ_SEC_END(sec_gn, 10)
-        if (gw == 0) { OQ_EV(7, s) }
+        if (fw == 0) { OQ_EV(9, i) }
+        ++next_tile;
+        advance(sl0, j0, BC);
       }
     }
   } else {
     // ------------------------------- compute warps -------------------------------
-    const int group = warp / WARPS_PER_TILE, q = warp & 3, colpart = (warp % WARPS_PER_TILE) >> 2;
+    const int q = warp & 3, colpart = warp >> 2;
     const int n = q * 32 + lane;                     // row of the tile = tensor-memory lane = pair
     const int t = n % TOK;
     const Poly2<(1 << (BITS - 1)) - 1> poly(p.poly);
     constexpr float blk_f = (float)BLK;
     const float inv_sqrt_h = rsqrtf(blk_f);
     const uint32_t tmem_thr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(colpart * (32 * PIECES));
+    int next_norm = 0;
     int sl0 = 0, j0 = 0;                             // first chunk of tile i
-    advance(sl0, j0, group * BC);
-    for (int i = group; i < ntiles; i += GROUPS, advance(sl0, j0, GROUPS * BC)) {
+    for (int i = 0; i < ntiles; ++i, advance(sl0, j0, BC)) {
       int sl = sl0, j = j0;
       advance(sl, j, n / TOK);
       const int row = ((int)blockIdx.x + sl * stride) * TOK + t;
       const bool valid = sl < nsl && row < p.rows;
       const int sl_last = tile_last_slab(sl0, j0);
-      warp_wait(bar(B_NORM + (sl_last & (NORM_RING - 1))), (uint32_t)(sl_last / NORM_RING) & 1u, WAIT_NORM);
-      const float s = s_norm[(min(sl, nsl - 1) & (NORM_RING - 1)) * 8 + t];
+      // norms of the slabs that this tile is the first to touch: the diagonal of the Gram matrix, added up over the
+      // 16 row groups in a fixed order (4 per lane quarter by shuffles, the 4 quarters by every reader)
+      for (; next_norm <= sl_last; ++next_norm) {
+        const int s = next_norm;
+        float* part = s_part + (s & (NORM_RING - 1)) * 32;
+        if (colpart == 0) {
+          warp_wait(bar(B_GRAMRDY), (uint32_t)s & 1u, WAIT_GRAM);
+          if (warp == 0) { OQ_EV(6, s) }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          uint32_t v[32];
+          tmem_load32(tmem + ((uint32_t)(q * 32) << 16) + GRAM_COL + (uint32_t)q * 32u, v);
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_GRAMFREE)) : "memory");
+          // entry (lane, lane) of the warp's 32 x 32 diagonal block
+#pragma unroll
+          for (int hb = 16; hb >= 1; hb >>= 1) {
+            const bool up = (lane & hb) != 0;
+#pragma unroll
+            for (int e = 0; e < hb; ++e) v[e] = up ? v[e + hb] : v[e];
+          }
+          float dsum = __uint_as_float(v[0]);
+          dsum += __shfl_xor_sync(0xffffffffu, dsum, 8);
+          dsum += __shfl_xor_sync(0xffffffffu, dsum, 16);
+          if (lane < 8) part[q * 8 + lane] = dsum;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(COMPUTE_WARPS * 32) : "memory");
+        if (warp == 0 && lane < TOK) {
+          float tot = 0.f;
+#pragma unroll
+          for (int qq = 0; qq < 4; ++qq)
+#pragma unroll
+            for (int hh = 0; hh < SUBS; ++hh) tot += part[qq * 8 + hh * TOK + lane];
+          const float nrm = sqrtf(tot);
+          const int orow = ((int)blockIdx.x + s * stride) * TOK + lane;
+          if (orow < p.rows) {
+            if (p.bf16_norm) reinterpret_cast<__nv_bfloat16*>(p.out_norm)[orow] = __float2bfloat16_rn(nrm);
+            else reinterpret_cast<float*>(p.out_norm)[orow] = nrm;
+          }
+          OQ_EV(7, s)
+        }
+      }
+      float tot = 0.f;
+      {
+        const float* part = s_part + (min(sl, nsl - 1) & (NORM_RING - 1)) * 32;
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq)
+#pragma unroll
+          for (int hh = 0; hh < SUBS; ++hh) tot += part[qq * 8 + hh * TOK + t];
+      }
+      const float s = sqrtf(tot);
       // |z| / (sqrt(h) (s + eps) clamp) with z the unnormalised block transform
       const float kappa = 1.0f / (sqrtf(blk_f) * (s + 1e-10f) * p.poly.clamp);
       const uint32_t slot = (uint32_t)i % 3u;
@@ -499,7 +451,7 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
         uint32_t vb[32];
         tmem_load32(tmem_thr + slot * 128u + 32u * piece, vb);
         if (piece == PIECES - 1) {
-          // the accumulator may be overwritten as soon as the warps of this group have read it
+          // the accumulator may be overwritten as soon as the compute warps have read it
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
           __syncwarp();
           if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar(B_ACCFREE + slot)) : "memory");
@@ -519,7 +471,7 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(vb[e]);
           const int cq = colpart * PIECES + piece;
-#if !defined(OQ_RQMM_TIMING) && !defined(OQ_RQMM_TRACE)
+#ifndef OQ_RQMM_TRACE
           if (p.dbg != nullptr) {
             float* d = p.dbg + (size_t)row * p.dim + j * 128 + cq * 32;
 #pragma unroll
@@ -540,14 +492,6 @@ __global__ void __launch_bounds__(rqmm::THREADS, 1) rq_mm_kernel(const RqMmParam
       if (warp == 0) { OQ_EV(11, i) }
     }
   }
-#ifdef OQ_RQMM_TIMING
-  if (lane == 0 && p.dbg != nullptr) {
-    long long* out = reinterpret_cast<long long*>(p.dbg) + ((size_t)blockIdx.x * 32 + warp) * 16;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) out[i] = tw[i];
-    out[15] = clock64() - t_begin;
-  }
-#endif
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();

@@ -19,11 +19,9 @@ struct RqMmParams {
   int nb;                   // dim / 128
   int seg_rows;             // 16-byte rows per segment of the slab buffer (a multiple of 16; 16 segments)
   int pad_rows;             // unused rows at the end of every segment
-  int nstages;              // staging ring: 2 or 3 stages
   int tab_smem;             // 1: the gather table is copied to shared memory
   int mask_smem;            // 1: the sign masks are copied to shared memory
   int bf16_norm;            // 1: norms stored as bf16 (weights), 0: fp32 (activations)
-  int desc_swap;            // test switch: exchange the two stride fields of the MN-major descriptors
   int* status;
 };
 

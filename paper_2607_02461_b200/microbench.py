@@ -5,6 +5,7 @@
     python -m paper_2607_02461_b200.microbench sweep [--quick]     # rotate+quantize bandwidth sweep
     python -m paper_2607_02461_b200.microbench adaln --tokens 1 --dim 3072 --m 18432   # AdaLN INT4 projection
     python -m paper_2607_02461_b200.microbench step --shape wan --bits-a 6             # whole block step, W4A6 or W4A4
+    python -m paper_2607_02461_b200.microbench ks --tokens 512 --dim 3072              # KS distance of rotated coordinates to f_d
 
 Inputs are synthetic and generated on the GPU (normal values, per-token log-uniform scale, 1% of the
 channels multiplied by 30); these runs time the kernels, parity is covered by the tests.
@@ -117,9 +118,37 @@ def run_step(shape, ba, bw, iters, split_qkv=False):
             "tflops_best": fl / best / 1e9}
 
 
+def run_ks(n, d, blocks):
+    """Diagnostic in the spirit of the paper's KS-distance figure: how close the coordinates of the rotated, normalised
+    tokens come to the marginal f_d that the codebook was fitted to (Eq. 2), per block size and with / without the
+    synthetic channel outliers.  Kolmogorov-Smirnov distance of each token's d coordinates to the cdf
+    F_d(t) = 1/2 + sgn(t) I_{t^2}(1/2, (d-1)/2) / 2, summarised over the tokens.  Uses the rotated values that
+    oq_rotate_quantize_act exports for the tests."""
+    import numpy as np
+    from scipy.special import betainc
+    out = []
+    g = torch.Generator(device="cuda").manual_seed(1)
+    plain = torch.randn((n, d), device="cuda", generator=g).to(torch.bfloat16)
+    for name, X in (("outliers_x30", gen_x(n, d)), ("gaussian", plain)):
+        for block in blocks:
+            if d % block:
+                continue
+            rot, cb = B.oq_make_rpbh(d, block, 0), B.oq_build_codebook(d, 4)
+            z = torch.empty((n, d), dtype=torch.float32, device="cuda")
+            _, s = B.oq_rotate_quantize_act(X, rot, cb, dbg_rotated=z)
+            t = np.sort((z / (s[:, None] + 1e-10)).double().cpu().numpy(), axis=1)
+            cdf = 0.5 + 0.5 * np.sign(t) * betainc(0.5, (d - 1) / 2.0, t * t)
+            i = np.arange(1, d + 1)[None, :] / d
+            ks = np.maximum(np.abs(cdf - i), np.abs(cdf - (i - 1.0 / d))).max(axis=1)
+            out.append({"kernel": "ks_distance", "input": name, "tokens": n, "dim": d, "block": block,
+                        "ks_median": float(np.median(ks)), "ks_max": float(ks.max()),
+                        "ks_of_a_perfect_sample": float(0.87 / np.sqrt(d))})
+    return out
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("mode", choices=["rq", "gemm", "sweep", "adaln", "step"])
+    ap.add_argument("mode", choices=["rq", "gemm", "sweep", "adaln", "step", "ks"])
     ap.add_argument("--tokens", type=int, default=17776)
     ap.add_argument("--dim", type=int, default=3072)
     ap.add_argument("--m", type=int, default=9216)
@@ -142,6 +171,9 @@ def main(argv=None):
         print(json.dumps(run_gemm(a.tokens, a.dim, a.m, a.bits_a, a.bits_w, a.iters, a.levels)))
     elif a.mode == "step":
         print(json.dumps(run_step(a.shape, a.bits_a, a.bits_w, a.iters, a.split_qkv)))
+    elif a.mode == "ks":
+        for r in run_ks(a.tokens, a.dim, [64, 128, 256, 1024]):
+            print(json.dumps(r))
     elif a.mode == "adaln":
         print(json.dumps(run_adaln(a.tokens, a.dim, a.m, a.iters)))
     else:

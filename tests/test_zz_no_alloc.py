@@ -42,6 +42,57 @@ def test_noalloc_matches_ordinary_path_on_two_calls_in_a_row():
         assert rel.item() <= 1e-5 and torch.equal(got32, want32)
 
 
+@pytest.mark.parametrize("d,bits", [(2048, 4), (3072, 3)])
+def test_noalloc_back_to_back_on_the_tensor_core_path_without_allocating(d, bits):
+    """The widths the benchmarks use run the tensor-core rotate+quantize kernel, launched with programmatic dependent
+    launch: three calls in a row on one stream, no synchronisation in between, all sharing the one scratch array (every
+    rotate+quantize overwrites what the GEMM before it reads).  Each must equal the two-call path bit for bit, and the
+    device's free memory must not move while they run."""
+    import torch
+    m = 776
+    rot, cb = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, bits)
+    assert B.oq_rq_plan(rot, cb)[0] == 3
+    wq, wr = B.oq_quantize_weights(_dev(synth.weights(m, d, 2100 + bits)), rot, cb)
+    Xs = [_dev(synth.activations(n, d, 30 + k)) for k, n in enumerate((513, 200, 1000))]
+    wants = []
+    for X in Xs:
+        xq, xs = B.oq_rotate_quantize_act(X, rot, cb)
+        wants.append(B.oq_qlinear(xq, xs, cb, wq, wr, cb, d))
+    outs = [torch.full((X.shape[0], m), float("nan"), dtype=torch.bfloat16, device="cuda") for X in Xs]
+    B.oq_linear_forward_noalloc(Xs[0], rot, cb, wq, wr, cb, outs[0])          # warm: first call on the device does the set-up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for X, out in zip(Xs, outs):
+        B.oq_linear_forward_noalloc(X, rot, cb, wq, wr, cb, out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert B.oq_device_status() == 0
+    for k, (got, want) in enumerate(zip(outs, wants)):
+        assert torch.equal(got, want), f"call {k}"
+
+
+def test_status_words_are_both_read_and_cleared():
+    """A time-out recorded in the library's own status word must not hide (or leave behind) one in the scratch array's
+    word, and the other way round: after one oq_device_status call both are clear and the next layer call is valid."""
+    import torch
+    d, m = 1024, 64
+    rot, cb = B.oq_make_rpbh(d, 128, 0), B.oq_build_codebook(d, 4)
+    wq, wr = B.oq_quantize_weights(_dev(synth.weights(m, d, 3)), rot, cb)
+    X = _dev(synth.activations(40, d, 4))
+    out = torch.empty((40, m), dtype=torch.bfloat16, device="cuda")
+    B.oq_linear_forward_noalloc(X, rot, cb, wq, wr, cb, out)                   # the scratch word exists now
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    B.oq_selftest_bounded_wait()                                              # a wait that simply runs out: code 9
+    assert B.oq_device_status() == 9
+    assert B.oq_device_status() == 0
+    B.oq_linear_forward_noalloc(X, rot, cb, wq, wr, cb, out)
+    xq, xs = B.oq_rotate_quantize_act(X, rot, cb)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.equal(out, B.oq_qlinear(xq, xs, cb, wq, wr, cb, d))
+
+
 def test_noalloc_rejects_what_does_not_fit_and_unprepared_handles():
     import torch
     d = 1024
