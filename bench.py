@@ -34,10 +34,13 @@ WORKLOADS = {
     "flux_w3a3": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 3, 3, 128),
     "flux_w2a4": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 2, 4, 128),
     "wan_w4a4": (synth.WAN_TOKENS, synth.WAN_LAYERS, 4, 4, 128),
+    # W4A6 (the paper's video setting): 64 activation levels travel as a bf16 level matrix between the two kernels
+    "flux_w4a6": (synth.FLUX_TOKENS, synth.FLUX_LAYERS, 4, 6, 128),
+    "wan_w4a6": (synth.WAN_TOKENS, synth.WAN_LAYERS, 4, 6, 128),
     "single_w4a4": (256, [("linear", 1024, 1024)], 4, 4, 128),
 }
-EXTRA_WORKLOADS = ["wan_w4a4", "flux_w3a3", "flux_w2a4"]      # measured after the headline workload, same process
-CONFIG_INDEX = {"single_w4a4": 0, "flux_w4a4": 1, "flux_w3a3": 1, "flux_w2a4": 2, "wan_w4a4": 3}
+EXTRA_WORKLOADS = ["wan_w4a4", "flux_w3a3", "flux_w2a4", "wan_w4a6"]      # measured after the headline workload, same process
+CONFIG_INDEX = {"single_w4a4": 0, "flux_w4a4": 1, "flux_w3a3": 1, "flux_w2a4": 2, "wan_w4a4": 3, "flux_w4a6": 1, "wan_w4a6": 3}
 METRIC = "qlinear effective TFLOP/s (whole step: rotate+quantize and codebook GEMM)"
 
 
@@ -51,6 +54,8 @@ def peaks():
 
 
 def rq_bytes(n, d, bits):
+    if bits == 6:
+        return 2 * n * d + 2 * n * d + 4 * n              # bf16 row in, bf16 level matrix + fp32 norm out
     return 2 * n * d + n * d * bits // 8 + 4 * n          # bf16 row in, packed indices + fp32 norm out
 
 
@@ -280,7 +285,8 @@ def prepare_workload(B, workload, dev, rank, host_copies):
         else:
             l["X"] = to_dev(xb)
         l["wq"], l["wr"] = B.oq_quantize_weights(to_dev(wb), rot, cbw)
-        l["xq"] = torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device=dev)
+        l["xq"] = (torch.empty((tokens, d), dtype=torch.bfloat16, device=dev) if ba == 6
+                   else torch.empty((tokens, B.oq_packed_bytes(tokens, d, ba)[1]), dtype=torch.uint8, device=dev))
         l["xs"] = torch.empty(tokens, dtype=torch.float32, device=dev)
         l["Y"] = torch.empty((tokens, m), dtype=torch.bfloat16, device=dev)
         L.append(l)
@@ -298,10 +304,16 @@ def time_workload(B, L, workload, steps, warmup, flush, world, dev, sampler_fact
         for l in L:
             if events is not None:
                 e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
-            B.oq_rotate_quantize_act(l["X"], l["rot"], l["cba"], out_idx=l["xq"], out_norm=l["xs"])
+            if ba == 6:
+                B.oq_rotate_quantize_act_levels(l["X"], l["rot"], l["cba"], out=l["xq"], out_norm=l["xs"])
+            else:
+                B.oq_rotate_quantize_act(l["X"], l["rot"], l["cba"], out_idx=l["xq"], out_norm=l["xs"])
             if events is not None:
                 e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
-            B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+            if ba == 6:
+                B.oq_qlinear_levels(l["xq"], l["xs"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+            else:
+                B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
         if events is not None:
             e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
 
@@ -414,9 +426,14 @@ def sustained_gemm(B, L, workload, dev, sampler_factory, seconds=2.0):
     tokens = WORKLOADS[workload][0]
     flops = sum(2 * tokens * l["m"] * l["d"] for l in L)
 
+    ba = WORKLOADS[workload][3]
+
     def gemms():
         for l in L:
-            B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+            if ba == 6:
+                B.oq_qlinear_levels(l["xq"], l["xs"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
+            else:
+                B.oq_qlinear(l["xq"], l["xs"], l["cba"], l["wq"], l["wr"], l["cbw"], l["d"], out=l["Y"])
     gemms(); torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record(); gemms(); b.record(); torch.cuda.synchronize()
@@ -525,7 +542,7 @@ def run_ours(args):
                    "per_kernel_timing": f"{r['inst_steps']} more steps right after the timed region with a CUDA event "
                                         f"between all kernels ({r['inst_ms']:.4f} ms per step: events between kernels "
                                         f"suspend programmatic dependent launch)"},
-        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel", "achieved": r["gemm"]["achieved"],
+        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel" + (" (levels form)" if ba == 6 else ""), "achieved": r["gemm"]["achieved"],
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": r["gemm"]["frac"],
                      "traffic": traffic.get("qlinear_bytes_per_step"), "traffic_source": traffic_source,
                      "peak_source": f"{pk['source']} burst (sustained {pk['bf16_tflops_sustained']})",
@@ -570,7 +587,7 @@ def run_ours(args):
         out["workloads"] = extra
         out["rq_sweep"] = rq_sweep(B, flush, dev)
         out["device_status_after_extras"] = B.oq_device_status()
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and ba != 6:      # (the oracle's 64-level codebooks take minutes each)
         stepf, flops, desc = oracle_sample(args.workload)
         stepf()
         t0 = time.perf_counter(); reps = 0
