@@ -217,3 +217,53 @@ def test_argument_checks_of_the_newer_entry_points_need_no_device():
     assert L.oq_adaln_quantize_weights(null, 32, 96, 96, null, null, null) == 2
     assert B.oq_adaln_packed_bytes(32, 128) == (32 * 128 // 2, 2 * 32 * 128 // 64)
     assert B.oq_forward_workspace_bytes(10, 3072, 16, 6) > B.oq_forward_workspace_bytes(10, 3072, 16, 4)
+
+
+def test_handles_and_errors_from_several_threads():
+    """Handles may be built and used from several host threads at once; oq_last_error is per thread."""
+    import threading
+    results, errors = {}, []
+
+    def work(k):
+        try:
+            cb = B.oq_build_codebook(1024 + 128 * k, 4)
+            rot = B.oq_make_rpbh(1024 + 128 * k, 128, k)
+            results[k] = (cb.centroids.copy(), rot.perm.copy(), B.oq_rq_plan(rot, cb)[0])
+            try:
+                B.oq_make_rpbh(100 + k, 64, 0)            # 64 does not divide 100 + k: an error on this thread only
+            except B.OqError as e:
+                results[("err", k)] = str(e)
+        except Exception as e:      # pragma: no cover
+            errors.append(repr(e))
+
+    ts = [threading.Thread(target=work, args=(k,)) for k in range(6)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    assert not errors
+    for k in range(6):
+        cb = B.oq_build_codebook(1024 + 128 * k, 4)
+        rot = B.oq_make_rpbh(1024 + 128 * k, 128, k)
+        assert np.array_equal(results[k][0], cb.centroids) and np.array_equal(results[k][1], rot.perm)
+        assert ("err", k) in results and results[("err", k)]
+
+
+def test_reference_arm_prints_the_contract_keys():
+    """`bench.py --impl reference` (the CPU oracle timed on a bounded sample) prints one JSON line with the keys the
+    benchmark contract asks for."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0",
+                          "--workload", "single_w4a4"], capture_output=True, text=True, timeout=600, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = json.loads([l for l in res.stdout.splitlines() if l.startswith("{")][-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["value"] > 0 and line["config"]["workload"] == "single_w4a4"
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
