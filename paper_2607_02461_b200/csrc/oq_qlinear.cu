@@ -37,7 +37,7 @@ constexpr uint32_t PA_BYTES = 2 * ATOM_BYTES, PB_BYTES = 2 * ATOM_BYTES;
 constexpr uint32_t PSTAGE_BYTES = PA_BYTES + PB_BYTES;                 // 64 KB
 constexpr int EPI_THREADS = 128;
 constexpr int PTHREADS = DECODE_THREADS + EPI_THREADS + 64;   // 16 decode warps, 4 epilogue warps, 1 MMA warp, 1 TMA warp
-constexpr size_t PSMEM_BYTES = PSTAGES * PSTAGE_BYTES + 1024 + 256;
+constexpr size_t PSMEM_BYTES = PSTAGES * PSTAGE_BYTES + 1024 + 256 + 2048;   // tiles, alignment slack, barriers, the epilogue warps' weight norms
 // Activations as bf16 levels: the TMA-fed activation tiles have a ring of their own, one stage deeper than the
 // weights' (their latency is the L2 round trip of a copy that can only be requested once its buffer is free; the
 // decoders hide theirs by holding the next stage's packed words in registers).
@@ -380,11 +380,21 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
   } else if (warp >= DECODE_THREADS / 32) {
     // ------------------------------- epilogue warps (4 per CTA) -------------------------------
     const int q = warp & 3;                          // TMEM lane quarter of this warp
+    // (packed form) the weight norms r' of the tile's 256 columns, one copy per warp, fetched before the warp waits for
+    // the accumulator so that the epilogue of a pair's last tile does not wait for them chunk by chunk
+    uint4* wn_s = reinterpret_cast<uint4*>(smem + PSTAGES * PSTAGE_BYTES + 256) + q * 32;
     uint32_t lt = 0;
     for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
       const uint32_t buf = lt & 1;
       const int n0 = (DENSE_A ? tile / tiles_m : tile % tiles_n) * 256 + (int)rank * 128;
       const int i0 = (DENSE_A ? tile % tiles_m : tile / tiles_n) * 256;
+      if constexpr (!DENSE_A) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i0 + lane * 8 < m) v = __ldg(reinterpret_cast<const uint4*>(w_norm + i0 + lane * 8));
+        __syncwarp();                                  // the other lanes have read the previous tile's copy
+        wn_s[lane] = v;
+        __syncwarp();
+      }
       if (lane == 0) mbar_wait(accfull0 + 8 * buf, (lt >> 1) & 1, abort_flag, status, WAIT_ACC_FULL);
       __syncwarp();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -400,7 +410,7 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
             for (int g8 = 0; g8 < 4; ++g8) {
               const int i = i0 + c * 32 + g8 * 8;
               if (i < m) {
-                const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));
+                const uint4 rn = DENSE_A ? __ldg(reinterpret_cast<const uint4*>(w_norm + i)) : wn_s[c * 4 + g8];
                 const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
                 float y[8];
 #pragma unroll
@@ -424,7 +434,7 @@ qlinear_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const uint32_t* 
             const int i = i0 + c * 32 + g8 * 8;
             pk[g8] = make_uint4(0u, 0u, 0u, 0u);
             if (i < m) {                               // (uniform over the warp)
-              const uint4 rn = __ldg(reinterpret_cast<const uint4*>(w_norm + i));
+              const uint4 rn = DENSE_A ? __ldg(reinterpret_cast<const uint4*>(w_norm + i)) : wn_s[c * 4 + g8];
               const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
               float y[8];
 #pragma unroll
