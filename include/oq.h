@@ -25,7 +25,8 @@
  *     numbered 0 .. 2^bits-1 in ascending order of the level, in rotated-coordinate order).
  *   - There is no CPU fallback: a call that needs the GPU fails with OQ_ERR_CUDA if no device is usable.
  *   - Threads: handles may be shared between host threads (first-use uploads are serialised inside the library);
- *     oq_last_error() is per thread; oq_debug_select_rq_kernel is a process-wide test switch and not thread-safe.
+ *     oq_last_error() is per thread; oq_debug_select_rq_kernel and oq_debug_select_gemm_kernel are process-wide test
+ *     switches and not thread-safe.
  */
 #ifndef OQ_H_
 #define OQ_H_
@@ -304,6 +305,15 @@ int oq_rq_plan(const oq_rpbh* rot, const oq_codebook* cb, int* kernel, int* rows
  * it measured slower).  A selected kernel that does not support the shape falls back.  All of them compute the same
  * function; the parity tests run each of them.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
 int oq_debug_select_rq_kernel(int which);
+
+/* Test helper: selects the kernel behind oq_qlinear (and the calls built on it) for the following calls of this
+ * process: 0 = choose by output type (default: kernel 2 for bf16 output, kernel 1 for fp32 output), 1 = both operands
+ * decoded into shared memory, two accumulators in tensor memory (the epilogue of a tile overlaps the next tile),
+ * 2 = the activation operand decoded into tensor memory (tcgen05.st; tcgen05.mma takes A from there), one accumulator,
+ * the output tile staged in shared memory; bf16 output only, fp32 output falls back to kernel 1.  Both compute the
+ * same sums in the same order: their outputs are bit-identical (Sec. 4.3, Eq. 6, Eq. 8).  oq_qlinear_levels always
+ * runs the shared-memory kernel.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
+int oq_debug_select_gemm_kernel(int which);
 
 const char* oq_last_error(void);
 const char* oq_version(void);

@@ -50,6 +50,7 @@ def lib():
             "oq_device_status": (i, [C.POINTER(i)]),
             "oq_selftest_bounded_wait": (i, [vp]),
             "oq_debug_select_rq_kernel": (i, [i]),
+            "oq_debug_select_gemm_kernel": (i, [i]),
             "oq_rq_plan": (i, [vp, vp, C.POINTER(i), C.POINTER(i), C.POINTER(i), C.POINTER(sz)]),
             "oq_rotate_quantize_act_levels": (i, [vp, i, i, i, vp, vp, vp, i, vp, vp, vp, vp]),
             "oq_decode_levels": (i, [vp, i, i, vp, vp, i, vp]),
@@ -266,6 +267,10 @@ def oq_rq_plan(rot, cb):
 
 def oq_debug_select_rq_kernel(which):
     _check(lib().oq_debug_select_rq_kernel(int(which)))
+
+
+def oq_debug_select_gemm_kernel(which):
+    _check(lib().oq_debug_select_gemm_kernel(int(which)))
 
 
 def oq_rotate_quantize_act_levels(X, rot, cb_a, out=None, out_norm=None, want_idx=False, dbg_rotated=None):

@@ -35,9 +35,16 @@ def run_case(n, m, d, ba, bw, block=128, seed=0, xseed=1000, wseed=2000, end_to_
     y32 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out_dtype=torch.float32)
     y16 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
     y16b = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+    # the two GEMM kernels (activation operand in shared memory / in tensor memory) add the same products in the same order
+    B.oq_debug_select_gemm_kernel(1)
+    y16_smem = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+    B.oq_debug_select_gemm_kernel(2)
+    y16_tmem = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+    B.oq_debug_select_gemm_kernel(0)
     torch.cuda.synchronize()
     assert B.oq_device_status() == 0
     assert torch.equal(y16, y16b)                                          # run-to-run determinism
+    assert torch.equal(y16, y16_tmem) and torch.equal(y16_smem, y16_tmem)
     # operand-exact mode: decode the GPU's own packed operands on the CPU, fp64 product
     ia = B.oq_unpack_indices(xq, n, d, ba).cpu().numpy()
     iw = B.oq_unpack_indices(wq, m, d, bw).cpu().numpy()

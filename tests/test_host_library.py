@@ -166,6 +166,11 @@ def test_rotate_quantize_plan_rejects_mismatched_handles():
     with pytest.raises(B.OqError) as e:
         B.oq_debug_select_rq_kernel(7)
     assert e.value.code == 1
+    with pytest.raises(B.OqError) as e:
+        B.oq_debug_select_gemm_kernel(3)
+    assert e.value.code == 1
+    for k in (1, 2, 0):
+        B.oq_debug_select_gemm_kernel(k)
     # a width that is not a multiple of 128 has no fast path at all
     with pytest.raises(B.OqError) as e:
         B.oq_rq_plan(B.oq_make_rpbh(192, 64, 0), B.oq_build_codebook(192, 4))
