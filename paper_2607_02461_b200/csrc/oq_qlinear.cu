@@ -514,7 +514,7 @@ constexpr uint32_t TB_BYTES = pair::PB_BYTES;                      // 32 KB of w
 constexpr uint32_t STAGING_OFF = TSTAGES * TB_BYTES;               // 128 KB
 constexpr uint32_t STAGING_WARP = 32 * 512;                        // 32 rows x 256 bf16 per epilogue warp
 constexpr uint32_t TBAR_OFF = STAGING_OFF + 4 * STAGING_WARP;      // 192 KB
-constexpr size_t TSMEM_BYTES = TBAR_OFF + 1024 + 256 + 2048;
+constexpr size_t TSMEM_BYTES = TBAR_OFF + 1024 + 256 + 4096;       // + alignment slack, barriers, the epilogue warps' weight norms (fp32)
 constexpr int TTHREADS = DECODE_THREADS + pair::EPI_THREADS + 32;  // 16 decode warps, 4 epilogue warps, 1 MMA warp
 constexpr uint32_t A_COL0 = 256;                                   // columns 0..255: the accumulator
 }  // namespace pairt
@@ -597,8 +597,9 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
   } else if (warp >= DECODE_THREADS / 32) {
     // ------------------------------- epilogue warps (4 per CTA) -------------------------------
     const int q = warp & 3;                          // TMEM lane quarter of this warp
-    uint4* wn_s = reinterpret_cast<uint4*>(smem + TBAR_OFF + 256) + q * 32;     // weight norms of the tile's 256 columns
+    float* wn_s = reinterpret_cast<float*>(smem + TBAR_OFF + 256) + q * 256;     // weight norms r' of the tile's 256 columns, fp32
     unsigned char* stage_w = smem + STAGING_OFF + (uint32_t)q * STAGING_WARP;   // this warp's 32 rows x 512 bytes
+    const uint32_t acc_thr = tmem + ((uint32_t)(q * 32) << 16);
     uint32_t lt = 0;
     for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
       const int n0 = (tile % tiles_n) * 256 + (int)rank * 128;
@@ -607,7 +608,10 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (i0 + lane * 8 < m) v = __ldg(reinterpret_cast<const uint4*>(w_norm + i0 + lane * 8));
         __syncwarp();                                  // the other lanes have read the previous tile's copy
-        wn_s[lane] = v;
+        reinterpret_cast<float4*>(wn_s)[2 * lane] = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                                                                  __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+        reinterpret_cast<float4*>(wn_s)[2 * lane + 1] = make_float4(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u),
+                                                                      __uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
         __syncwarp();
       }
       const int trow = n0 + q * 32 + lane;
@@ -616,27 +620,33 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
       __syncwarp();
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       unsigned char* my_row = stage_w + (uint32_t)lane * 512u;
-#pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        uint32_t r[32];
-        tmem_load32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), r);
+      // 16 pieces of 16 columns; the load of a piece is in flight while the one before it is scaled, rounded and staged
+      auto stage16 = [&](const uint32_t (&r)[16], int pc) {
 #pragma unroll
-        for (int g8 = 0; g8 < 4; ++g8) {
-          const uint4 rn = wn_s[c * 4 + g8];
-          const uint32_t rw[4] = {rn.x, rn.y, rn.z, rn.w};
+        for (int g8 = 0; g8 < 2; ++g8) {
+          const float4 ra = reinterpret_cast<const float4*>(wn_s)[pc * 4 + g8 * 2], rb = reinterpret_cast<const float4*>(wn_s)[pc * 4 + g8 * 2 + 1];
+          const float rw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
           float y[8];
 #pragma unroll
-          for (int jj = 0; jj < 4; ++jj) {
-            y[2 * jj] = (__uint_as_float(r[g8 * 8 + 2 * jj]) * s) * __uint_as_float(rw[jj] << 16);
-            y[2 * jj + 1] = (__uint_as_float(r[g8 * 8 + 2 * jj + 1]) * s) * __uint_as_float(rw[jj] & 0xFFFF0000u);
-          }
+          for (int jj = 0; jj < 8; ++jj) y[jj] = (__uint_as_float(r[g8 * 8 + jj]) * s) * rw[jj];
           __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
           __nv_bfloat162 p2 = __floats2bfloat162_rn(y[4], y[5]), p3 = __floats2bfloat162_rn(y[6], y[7]);
           const uint4 pk = make_uint4(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1),
                                       *reinterpret_cast<uint32_t*>(&p2), *reinterpret_cast<uint32_t*>(&p3));
-          // 16-byte unit u = 4 c + g8 of the row sits at position u ^ lane
-          *reinterpret_cast<uint4*>(my_row + ((uint32_t)((c * 4 + g8) ^ lane) << 4)) = pk;
+          // 16-byte unit u = 2 pc + g8 of the row sits at position u ^ lane
+          *reinterpret_cast<uint4*>(my_row + ((uint32_t)((pc * 2 + g8) ^ lane) << 4)) = pk;
         }
+      };
+      uint32_t ra[16], rb[16];
+      tmem_load16_nowait(acc_thr, ra);
+#pragma unroll 1
+      for (int pc = 0; pc < 16; pc += 2) {
+        tmem_wait_ld();
+        tmem_load16_nowait(acc_thr + (uint32_t)(pc + 1) * 16u, rb);
+        stage16(ra, pc);
+        tmem_wait_ld();
+        if (pc + 2 < 16) tmem_load16_nowait(acc_thr + (uint32_t)(pc + 2) * 16u, ra);
+        stage16(rb, pc + 1);
       }
       // the accumulator has been read: the MMAs of the pair's next tile may overwrite it
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
