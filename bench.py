@@ -542,7 +542,7 @@ def run_ours(args):
                    "per_kernel_timing": f"{r['inst_steps']} more steps right after the timed region with a CUDA event "
                                         f"between all kernels ({r['inst_ms']:.4f} ms per step: events between kernels "
                                         f"suspend programmatic dependent launch)"},
-        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel" + (" (levels form)" if ba == 6 else ""), "achieved": r["gemm"]["achieved"],
+        "roofline": {"bound": "tensor", "kernel": "qlinear_pair_kernel (levels form)" if ba == 6 else "qlinear_pair_tmem_a_kernel", "achieved": r["gemm"]["achieved"],
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": r["gemm"]["frac"],
                      "traffic": traffic.get("qlinear_bytes_per_step"), "traffic_source": traffic_source,
                      "peak_source": f"{pk['source']} burst (sustained {pk['bf16_tflops_sustained']})",
