@@ -213,3 +213,29 @@ def test_whole_layer_with_the_papers_default_block(n, m, d, block):
     """Both operands rotated with the paper's default block (the largest power of two dividing the width): the rotation
     cancels in the product (Sec. 4.3) whatever the block, and the layer matches the oracle end to end."""
     run_case(n, m, d, 4, 4, block=block, seed=3)
+
+
+@pytest.mark.parametrize("ba,bw", [(4, 4), (3, 3), (2, 4)])
+def test_both_gemm_kernels_agree_over_several_tiles_per_sm_pair(ba, bw):
+    """156 output tiles on at most 74 SM pairs: every pair runs two or three tiles, so the kernel with the activation operand
+    in tensor memory reuses its single accumulator, its operand ring and its staging area; ragged last row and column tiles."""
+    import torch
+    n, m, d = 2990, 3304, 1024
+    rot = B.oq_make_rpbh(d, 128, 0)
+    cba, cbw = B.oq_build_codebook(d, ba), B.oq_build_codebook(d, bw)
+    xq, xs = B.oq_rotate_quantize_act(_dev(synth.activations(n, d, 1234)), rot, cba)
+    wq, wr = B.oq_quantize_weights(_dev(synth.weights(m, d, 2345)), rot, cbw)
+    try:
+        B.oq_debug_select_gemm_kernel(1)
+        y1 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+        B.oq_debug_select_gemm_kernel(2)
+        y2 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+        y2b = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+    finally:
+        B.oq_debug_select_gemm_kernel(0)
+    torch.cuda.synchronize()
+    assert B.oq_device_status() == 0
+    assert torch.equal(y1, y2) and torch.equal(y2, y2b)
+    # and against the fp32 output of kernel 1 rounded once
+    y32 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out_dtype=torch.float32)
+    assert torch.equal(y32.to(torch.bfloat16), y2)
