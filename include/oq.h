@@ -310,8 +310,10 @@ int oq_debug_select_rq_kernel(int which);
  * process: 0 = choose by output type (default: kernel 2 for bf16 output, kernel 1 for fp32 output), 1 = both operands
  * decoded into shared memory, two accumulators in tensor memory (the epilogue of a tile overlaps the next tile),
  * 2 = the activation operand decoded into tensor memory (tcgen05.st; tcgen05.mma takes A from there), one accumulator,
- * the output tile staged in shared memory; bf16 output only, fp32 output falls back to kernel 1.  Both compute the
- * same sums in the same order: their outputs are bit-identical (Sec. 4.3, Eq. 6, Eq. 8).  oq_qlinear_levels always
+ * the output tile staged in shared memory; bf16 output only, fp32 output falls back to kernel 1; 3 = kernel 2 with the
+ * tile order it otherwise uses only for large inputs (bands of 8 column tiles, chosen by the library when the packed
+ * activations exceed 32 MB).  All of them compute the same sums in the same order: their outputs are bit-identical
+ * (Sec. 4.3, Eq. 6, Eq. 8).  oq_qlinear_levels always
  * runs the shared-memory kernel.  Not thread-safe.  Returns OQ_OK or OQ_ERR_INVALID_ARG. */
 int oq_debug_select_gemm_kernel(int which);
 

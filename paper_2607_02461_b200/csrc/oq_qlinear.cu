@@ -164,14 +164,29 @@ __device__ __forceinline__ void dense_b_decode_loop(const uint32_t* __restrict__
   }
 }
 
+// Tile order of the kernel with the activation operand in tensor memory: bands of `width` column tiles; inside a band the
+// column tile varies fastest.  With width 1 the row tile varies fastest over the whole matrix (the pairs that run together
+// share one weight tile and read npairs different activation tiles: fine while the packed activations stay in L2).  With
+// width 8 they work on ~npairs / 8 row tiles x 8 column tiles, so both packed operands of a wave are a few MB: chosen by
+// the launcher when the packed activations are too large to stay in L2 next to the output stream (Wan-sized layers: +4 %).
+constexpr int TILE_BAND_WIDE = 8;
+__device__ __forceinline__ void banded_tile(int tile, int tiles_n, int tiles_m, int width, int& rt, int& ct) {
+  const int band = tile / (width * tiles_n);
+  const int c0 = band * width;
+  const int gc = min(width, tiles_m - c0);
+  const int r = tile - band * width * tiles_n;
+  rt = r / gc;
+  ct = c0 + r - rt * gc;
+}
+
 // Decode loop of one thread of the two-SM kernel: the thread owns one (row, 32-coordinate half) of this CTA's
 // 128 rows of ONE operand (IS_A: activations, else weights) and, per 128-coordinate stage, decodes the two
 // 32-coordinate pieces that fall into the stage's two swizzle atoms.
-template <int BITS, bool IS_A, uint32_t STAGE_STRIDE = pair::PSTAGE_BYTES, int NSTAGES = pair::PSTAGES, uint32_t B_OFF = pair::PA_BYTES>
+template <int BITS, bool IS_A, uint32_t STAGE_STRIDE = pair::PSTAGE_BYTES, int NSTAGES = pair::PSTAGES, uint32_t B_OFF = pair::PA_BYTES, bool BANDED = false>
 __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ packed, int nrows, int dim, const Tables& t,
                                                  unsigned char* smem, uint32_t full0, uint32_t empty0, int t2,
                                                  uint32_t rank, int pair_id, int npairs, int ntiles, int tiles_n,
-                                                 int kblocks, volatile int* abort_flag, int* status) {
+                                                 int kblocks, volatile int* abort_flag, int* status, int tiles_m = 0, int band = 1) {
   using namespace pair;
   const int lane = threadIdx.x & 31;
   // Two ways to split a stage's 128 rows x 128 coordinates among 256 threads:
@@ -198,7 +213,9 @@ __device__ __forceinline__ void pair_decode_loop(const uint32_t* __restrict__ pa
   int f_tile = pair_id, f_kb = 0;
   const uint32_t* fsrc = nullptr;
   auto set_fetch_tile = [&](int tile) {
-    const int r0 = (IS_A ? (tile % tiles_n) : (tile / tiles_n)) * 256 + (int)rank * 128;
+    int rt = tile % tiles_n, ct = tile / tiles_n;
+    if constexpr (BANDED) banded_tile(tile, tiles_n, tiles_m, band, rt, ct);
+    const int r0 = (IS_A ? rt : ct) * 256 + (int)rank * 128;
     fsrc = packed + (size_t)min(r0 + row, nrows - 1) * pitch + sub * (CONTIG ? WPA : BITS);   // rows past the end re-read the last
   };
   auto fetch_next = [&]() {
@@ -523,7 +540,7 @@ template <int BITS_A, int BITS_W>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pairt::TTHREADS, 1)
 qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restrict__ a_norm, int n_tokens,
                            const uint32_t* __restrict__ Wq, const __nv_bfloat16* __restrict__ w_norm, int m, int dim,
-                           CodebookParams cba, CodebookParams cbw, __nv_bfloat16* __restrict__ Y, int ldy, int* status) {
+                           CodebookParams cba, CodebookParams cbw, __nv_bfloat16* __restrict__ Y, int ldy, int band, int* status) {
   using namespace pair;
   using namespace pairt;
   extern __shared__ unsigned char smem_dyn[];
@@ -602,8 +619,10 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
     const uint32_t acc_thr = tmem + ((uint32_t)(q * 32) << 16);
     uint32_t lt = 0;
     for (int tile = pair_id; tile < ntiles; tile += npairs, ++lt) {
-      const int n0 = (tile % tiles_n) * 256 + (int)rank * 128;
-      const int i0 = (tile / tiles_n) * 256;
+      int rt, ct;
+      banded_tile(tile, tiles_n, tiles_m, band, rt, ct);
+      const int n0 = rt * 256 + (int)rank * 128;
+      const int i0 = ct * 256;
       {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (i0 + lane * 8 < m) v = __ldg(reinterpret_cast<const uint4*>(w_norm + i0 + lane * 8));
@@ -676,7 +695,9 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
     int f_tile = pair_id, f_kb = 0;
     const uint32_t* fsrc = nullptr;
     auto set_fetch_tile = [&](int tile) {
-      const int r0 = (tile % tiles_n) * 256 + (int)rank * 128;
+      int rt, ct;
+      banded_tile(tile, tiles_n, tiles_m, band, rt, ct);
+      const int r0 = rt * 256 + (int)rank * 128;
       fsrc = Aq + (size_t)min(r0 + row, n_tokens - 1) * pitch + khalf * 2 * BITS_A;   // rows past the end re-read the last
     };
     auto fetch_next = [&]() {
@@ -720,8 +741,8 @@ qlinear_pair_tmem_a_kernel(const uint32_t* __restrict__ Aq, const float* __restr
   } else {
     // ------------------------------- decoders of the weights (8 warps) -------------------------------
     const Tables tw = make_tables(cbw);
-    pair_decode_loop<BITS_W, false, TB_BYTES, TSTAGES, 0u>(Wq, m, dim, tw, smem, full0, empty0, tid - 256, rank, pair_id, npairs,
-                                                            ntiles, tiles_n, kblocks, abort_flag, status);
+    pair_decode_loop<BITS_W, false, TB_BYTES, TSTAGES, 0u, true>(Wq, m, dim, tw, smem, full0, empty0, tid - 256, rank, pair_id, npairs,
+                                                                  ntiles, tiles_n, kblocks, abort_flag, status, tiles_m, band);
   }
   __syncwarp();
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -820,7 +841,8 @@ cudaError_t launch_pair(const CUtensorMap& tmap, int sms, cudaStream_t st, const
   return launch_dependent(k, 2 * pairs, pair::PTHREADS, smem_bytes, st, tmap, Aq, an, n, Wq, wn, m, dim, ca, cw, Y, ldy, status);
 }
 
-int g_gemm_kernel = 0;       // oq_debug_select_gemm_kernel: 0 by output type, 1 activation operand in shared memory, 2 in tensor memory
+int g_gemm_kernel = 0;       // oq_debug_select_gemm_kernel: 0 by output type, 1 activation operand in shared memory, 2 in tensor memory,
+                             // 3 in tensor memory with the wide tile bands at any size
 
 template <int BA, int BW>
 cudaError_t launch_pair_tmem_a(int sms, cudaStream_t st, const uint32_t* Aq, const float* an, int n, const uint32_t* Wq,
@@ -847,8 +869,10 @@ cudaError_t launch_pair_tmem_a(int sms, cudaStream_t st, const uint32_t* Aq, con
   int pairs = (dev >= 0 && dev < 64) ? max_pairs[dev].load(std::memory_order_relaxed) : sms / 2;
   if (pairs > sms / 2) pairs = sms / 2;
   if (pairs > ntiles) pairs = ntiles;
+  // (see banded_tile) packed activations above 32 MB: bands of 8 column tiles
+  const int band = (g_gemm_kernel == 3 || (size_t)n * dim * BA / 8 > ((size_t)32 << 20)) ? TILE_BAND_WIDE : 1;
   return launch_dependent(k, 2 * pairs, pairt::TTHREADS, smem_bytes, st, Aq, an, n, Wq, wn, m, dim, ca, cw,
-                          reinterpret_cast<__nv_bfloat16*>(Y), ldy, status);
+                          reinterpret_cast<__nv_bfloat16*>(Y), ldy, band, status);
 }
 
 template <int BA, int BW>
@@ -1019,7 +1043,7 @@ extern "C" int oq_qlinear(const void* Xq_idx, const float* Xq_norm, int n_tokens
 }
 
 extern "C" int oq_debug_select_gemm_kernel(int which) {
-  if (which < 0 || which > 2) return oq::fail(OQ_ERR_INVALID_ARG, "oq_debug_select_gemm_kernel: unknown kernel");
+  if (which < 0 || which > 3) return oq::fail(OQ_ERR_INVALID_ARG, "oq_debug_select_gemm_kernel: unknown kernel");
   oq::g_gemm_kernel = which;
   return OQ_OK;
 }

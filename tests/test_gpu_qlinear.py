@@ -40,11 +40,13 @@ def run_case(n, m, d, ba, bw, block=128, seed=0, xseed=1000, wseed=2000, end_to_
     y16_smem = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
     B.oq_debug_select_gemm_kernel(2)
     y16_tmem = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+    B.oq_debug_select_gemm_kernel(3)                                       # the tile order of large inputs
+    y16_band = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
     B.oq_debug_select_gemm_kernel(0)
     torch.cuda.synchronize()
     assert B.oq_device_status() == 0
     assert torch.equal(y16, y16b)                                          # run-to-run determinism
-    assert torch.equal(y16, y16_tmem) and torch.equal(y16_smem, y16_tmem)
+    assert torch.equal(y16, y16_tmem) and torch.equal(y16_smem, y16_tmem) and torch.equal(y16_band, y16_tmem)
     # operand-exact mode: decode the GPU's own packed operands on the CPU, fp64 product
     ia = B.oq_unpack_indices(xq, n, d, ba).cpu().numpy()
     iw = B.oq_unpack_indices(wq, m, d, bw).cpu().numpy()
@@ -231,11 +233,13 @@ def test_both_gemm_kernels_agree_over_several_tiles_per_sm_pair(ba, bw):
         B.oq_debug_select_gemm_kernel(2)
         y2 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
         y2b = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
+        B.oq_debug_select_gemm_kernel(3)               # 13 column tiles: one band of 8 and one of 5
+        y3 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d)
     finally:
         B.oq_debug_select_gemm_kernel(0)
     torch.cuda.synchronize()
     assert B.oq_device_status() == 0
-    assert torch.equal(y1, y2) and torch.equal(y2, y2b)
+    assert torch.equal(y1, y2) and torch.equal(y2, y2b) and torch.equal(y2, y3)
     # and against the fp32 output of kernel 1 rounded once
     y32 = B.oq_qlinear(xq, xs, cba, wq, wr, cbw, d, out_dtype=torch.float32)
     assert torch.equal(y32.to(torch.bfloat16), y2)

@@ -167,9 +167,9 @@ def test_rotate_quantize_plan_rejects_mismatched_handles():
         B.oq_debug_select_rq_kernel(7)
     assert e.value.code == 1
     with pytest.raises(B.OqError) as e:
-        B.oq_debug_select_gemm_kernel(3)
+        B.oq_debug_select_gemm_kernel(4)
     assert e.value.code == 1
-    for k in (1, 2, 0):
+    for k in (1, 2, 3, 0):
         B.oq_debug_select_gemm_kernel(k)
     # a width that is not a multiple of 128 has no fast path at all
     with pytest.raises(B.OqError) as e:
