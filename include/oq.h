@@ -125,7 +125,8 @@ int oq_quantize_weights(const void* W_bf16, int m, int dim, int ldw, const oq_rp
 
 /* Quantized linear layer on packed operands (the product W^' x^' of Sec. 4.3 with Eq. 6 and Eq. 8):
  *   Y[n][i] = s_n * r'_i * sum_k C_a[idxA[n][k]] * C_w[idxW[i][k]]
- * Levels are decoded to bf16 in shared memory, contracted on the tensor cores with fp32 accumulation,
+ * Levels are decoded to bf16 on the SM (weights into shared memory, activations into tensor or shared memory, see
+ * oq_debug_select_gemm_kernel), contracted on the tensor cores with fp32 accumulation,
  * and both norms are applied in the epilogue (acc * s_n * r'_i, two fp32 multiplies in that order, then
  * one rounding when Y is bf16).
  *   Xq_idx, Xq_norm  dev  as written by oq_rotate_quantize_act with cb_a
